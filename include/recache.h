@@ -1,0 +1,219 @@
+/*
+ * recache.h - C ABI of the resource-routed attention library (sm_100a).
+ *
+ * The four hot-path calls follow the problem statement of the ReCache paper
+ * (section "ReCache"): resources are encoded one by one with positions that
+ * restart inside each resource ("Resource-Wise Attention"); at request time the
+ * conversation sees, on every (layer, KV-head-group) route, only the resources
+ * that route exposes ("Structural Pruning", masks M_resource / M_context) and
+ * only their retained token fields ("Semantic Pruning"); the gather of those
+ * rows is the "request-local KV materialization" the paper counts inside TTFT
+ * (section "Evaluation Metrics", paragraph "Efficiency").
+ *
+ * Conventions that hold for every call
+ *  - Every tensor pointer is CALLER-OWNED DEVICE memory of the context's dtype
+ *    (float or bfloat16) unless the comment says otherwise.  The library keeps
+ *    no pointer past the call and frees nothing it was given.
+ *  - int32 index arrays (cu_seqlens, slots, tables ...) are DEVICE pointers.
+ *    Plain int arguments are host values: exact sizes or upper bounds used to
+ *    size launches.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls enqueue work and return
+ *    without synchronising.
+ *  - `workspace` is caller-owned device scratch of at least the number of bytes
+ *    the matching recache_*_workspace_bytes() query returns (256-byte aligned).
+ *    Its contents are undefined after the call.
+ *  - Return value: RECACHE_OK, or an error detected on the host BEFORE any
+ *    launch (null pointer, unsupported shape, capacity too small, CUDA launch
+ *    failure).  recache_last_error() gives the text.
+ *  - Errors only the device can see (an index outside its buffer, a position
+ *    past the rotary table, a route longer than the capacity given) never trap:
+ *    the offending access is skipped and a code is stored in the context's
+ *    device status word, read (and cleared) by recache_poll_status().
+ *
+ * Layouts (d = head_dim, G = n_kv_heads, Hq = n_q_heads, s = Hq / G; query head
+ * h reads KV group h / s)
+ *  - token-major activations:  q [tokens][Hq][d];  k, v [tokens][G][d]
+ *  - resource cache (one layer): k_cache, v_cache [G][pool_tokens][d]; resource
+ *    i occupies rows dst_slot[i] .. dst_slot[i] + D_i - 1 of every group
+ *  - packed route KV: [rows][d]; route r = request * G + group owns rows
+ *    route_cu[r] .. route_cu[r+1]-1
+ *  - paged KV: k_pages, v_pages [n_pages][page_tokens][d]; a page belongs to
+ *    one (sequence, group) item
+ *  - rotary embedding pairs element i with i + d/2; angle = pos * theta^(-2i/d)
+ */
+#ifndef RECACHE_H
+#define RECACHE_H
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RECACHE_API __attribute__((visibility("default")))
+#else
+#define RECACHE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RECACHE_OK = 0,
+  RECACHE_EINVAL = 1,       /* null pointer, negative size, bad enum */
+  RECACHE_ESHAPE = 2,       /* head counts / head_dim / sizes inconsistent */
+  RECACHE_EUNSUPPORTED = 3, /* valid but not implemented for this dtype/shape */
+  RECACHE_ENOMEM = 4,       /* workspace or capacity too small, allocation failed */
+  RECACHE_ECUDA = 5         /* a CUDA runtime/driver call failed */
+} recache_status;
+
+enum { RECACHE_F32 = 0, RECACHE_BF16 = 1 };
+enum { RECACHE_PACKED = 0, RECACHE_PAGED = 1 };
+
+/* Codes stored in the device status word (first error wins). */
+enum {
+  RECACHE_DEV_OK = 0,
+  RECACHE_DEV_BAD_SEQLENS = 1,  /* cu_seqlens / cu_q not monotone or past total */
+  RECACHE_DEV_BAD_SLOT = 2,     /* cache row outside [0, pool_tokens) */
+  RECACHE_DEV_OVERFLOW = 3,     /* route rows exceed row_capacity */
+  RECACHE_DEV_BAD_PAGE = 4,     /* page id outside [0, n_pages) or table too short */
+  RECACHE_DEV_NO_PAGES = 5,     /* free page list exhausted */
+  RECACHE_DEV_BAD_POS = 6       /* position outside [0, max_pos) */
+};
+
+typedef struct recache_ctx recache_ctx;
+
+typedef struct {
+  int32_t n_q_heads;   /* Hq */
+  int32_t n_kv_heads;  /* G; Hq % G == 0, Hq / G <= 8 */
+  int32_t head_dim;    /* 64 or 128 */
+  int32_t dtype;       /* RECACHE_F32 or RECACHE_BF16: storage of q/k/v/caches */
+  int32_t max_pos;     /* rotary table rows: every position must be < max_pos */
+  int32_t page_tokens; /* tokens per KV page (64) */
+  double rope_theta;
+} recache_desc;
+
+/* Creates a context on `device`: builds the cos/sin table (computed in double on
+ * the host, stored as float, max_pos * head_dim * 4 bytes on the device) and the
+ * device status word.  The only call that allocates device memory. */
+RECACHE_API recache_status recache_create(recache_ctx** out, const recache_desc* desc, int device);
+RECACHE_API void recache_destroy(recache_ctx* ctx);
+/* Text of the last host-side error of this context ("" if none). Host pointer,
+ * owned by the context. */
+RECACHE_API const char* recache_last_error(const recache_ctx* ctx);
+/* Synchronises `stream`, returns the device status word in *device_code and
+ * clears it. */
+RECACHE_API recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* device_code);
+
+/* Scratch sizes in bytes for the calls below (same size arguments). */
+RECACHE_API int64_t recache_encode_workspace_bytes(const recache_ctx* ctx, int32_t n_resources,
+                                       int32_t total_tokens, int32_t max_len);
+RECACHE_API int64_t recache_compact_workspace_bytes(const recache_ctx* ctx, int32_t n_requests,
+                                        int32_t total_listed);
+RECACHE_API int64_t recache_prefill_workspace_bytes(const recache_ctx* ctx, int32_t n_requests,
+                                        int32_t total_q, int32_t max_q);
+RECACHE_API int64_t recache_decode_workspace_bytes(const recache_ctx* ctx, int32_t batch,
+                                       int32_t max_res_pages, int32_t max_hist_pages);
+
+/*
+ * Resource-wise encoding (paper: "Resource-Wise Attention"; figure panel (a)).
+ * N resources are packed back to back; resource i is rows cu_seqlens[i] ..
+ * cu_seqlens[i+1]-1 and its token j has position j (0-based).  For every token
+ * j of resource i and query head h:
+ *     o[i,j,h] = sum_{j' <= j} softmax_j'( rope(q,j) . rope(k,j') / sqrt(d) ) v[j']
+ * with keys/values of the same resource only.  The rotated keys and the values
+ * are written to the cache rows dst_slot[i] + j.  Nothing computed for a
+ * resource depends on the other resources of the batch, their order or the
+ * launch: outputs and cache rows are bit-identical across compositions.
+ *   q [T][Hq][d], k/v [T][G][d] pre-rotation;  T = total_tokens (exact);
+ *   max_len >= every D_i;  dst_slot [N];  caches [G][pool_tokens][d];
+ *   out_o [T][Hq][d] of out_dtype (RECACHE_F32 or the context dtype).
+ * Empty resources (D_i = 0) are allowed.
+ */
+RECACHE_API recache_status recache_encode_resources(recache_ctx* ctx,
+    const void* q, const void* k, const void* v,
+    const int32_t* cu_seqlens, int32_t n_resources, int32_t total_tokens, int32_t max_len,
+    const int32_t* dst_slot, void* k_cache, void* v_cache, int64_t pool_tokens,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
+ * Route / keep-mask compaction = request-local KV materialisation (paper:
+ * "Structural Pruning", "Semantic Pruning", and the TTFT definition).
+ * Request b lists resources res_off[b] .. res_off[b+1]-1 (entries of res_slot /
+ * res_len, in request order).  Route r = b * G + g exposes, in this order, the
+ * listed resources with vis[g][listed index] != 0, and of each the cache rows
+ * slot + j (j ascending) with keep[slot + j] != 0.
+ *   keep [pool_tokens] uint8;  vis [G][total_listed] uint8 (this layer's routes)
+ * Outputs
+ *   route_cu  [B*G+1]  exclusive prefix of route lengths
+ *   route_len [B*G]    (optional, may be NULL) the lengths themselves
+ *   route_idx [row_capacity] cache row of every compacted row, packed order
+ *   mode RECACHE_PACKED: k_out/v_out [row_capacity][d] packed route KV
+ *   mode RECACHE_PAGED : k_out/v_out are page pools [n_pool_pages][page_tokens][d];
+ *        route r takes ceil(len_r / page_tokens) consecutive entries of
+ *        free_pages [n_free_pages], starting where route r-1 stopped; row n of
+ *        the route goes to page_table[r][n / page_tokens], slot n % page_tokens;
+ *        page_table [B*G][max_pages_per_route] is padded with -1.
+ * Indices are exact (stable order); gathered rows are byte copies.  A route with
+ * no visible resource or no kept token has length 0.
+ */
+RECACHE_API recache_status recache_compact_routes(recache_ctx* ctx,
+    const void* k_cache, const void* v_cache, int64_t pool_tokens,
+    const uint8_t* keep,
+    const int32_t* res_off, const int32_t* res_slot, const int32_t* res_len,
+    int32_t n_requests, int32_t total_listed,
+    const uint8_t* vis, int32_t mode,
+    int32_t* route_cu, int32_t* route_len, int32_t* route_idx, int64_t row_capacity,
+    void* k_out, void* v_out,
+    int32_t* page_table, int32_t max_pages_per_route,
+    const int32_t* free_pages, int64_t n_free_pages, int64_t n_pool_pages,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
+ * Routed prefill (paper: final mask of the architecture figure; routes in Omega
+ * use M_resource, the others M_context).  Query token t of request b has
+ * position q_pos0[b] + t.  For head h in group g, ONE softmax (scale 1/sqrt(d))
+ * runs over (i) all rows of route b*G+g in k_route/v_route (keys used as cached,
+ * no causal restriction) and (ii) conversation tokens t' <= t of the same
+ * request (keys rotated at their own positions).  A route of length 0 is plain
+ * causal self-attention of the conversation.
+ *   q [total_q][Hq][d], k_conv/v_conv [total_q][G][d] pre-rotation;
+ *   cu_q [B+1], q_pos0 [B];  max_q >= every request's length;
+ *   k_route/v_route packed [route_rows][d] with route_cu [B*G+1] (from compaction)
+ * Outputs
+ *   k_conv_out/v_conv_out [G][total_q][d]: rotated conversation keys / values,
+ *       head-major (the rows a later decode step keeps as history); required
+ *   out_o [total_q][Hq][d] of out_dtype.
+ */
+RECACHE_API recache_status recache_attend_prefill(recache_ctx* ctx,
+    const void* q, const void* k_conv, const void* v_conv,
+    const int32_t* cu_q, const int32_t* q_pos0,
+    int32_t n_requests, int32_t total_q, int32_t max_q,
+    const void* k_route, const void* v_route, const int32_t* route_cu, int64_t route_rows,
+    void* k_conv_out, void* v_conv_out,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
+ * Routed decode (paper: the same mask "during decoding"; the Attn. latency of
+ * the efficiency study).  One query token per sequence at position q_pos[b].
+ * Item it = b * G + g reads res_len[it] rows through res_page_table[it][*] and
+ * hist_len[it] rows through hist_page_table[it][*] (row n lives in page
+ * table[n / page_tokens], slot n % page_tokens); one softmax over both parts.
+ * If k_new/v_new ([B][G][d], pre-rotation) are given, the current token's
+ * rotated key and value are first written as history row hist_len[it]-1; pass
+ * NULL when the caller has appended them already.  hist_len >= 1 always.
+ *   q [B][Hq][d] pre-rotation;  out_o [B][Hq][d] of out_dtype.
+ */
+RECACHE_API recache_status recache_attend_decode(recache_ctx* ctx,
+    const void* q, const int32_t* q_pos, int32_t batch,
+    const void* k_new, const void* v_new,
+    void* k_pages, void* v_pages, int64_t n_pages,
+    const int32_t* res_page_table, int32_t max_res_pages, const int32_t* res_len,
+    const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RECACHE_H */

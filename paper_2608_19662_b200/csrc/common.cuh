@@ -1,0 +1,118 @@
+// Internal declarations shared by the translation units of librecache.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string>
+
+#include "recache.h"
+
+struct recache_ctx {
+  recache_desc desc;
+  int device;
+  float* cos_tab;     // [max_pos][d/2]
+  float* sin_tab;     // [max_pos][d/2]
+  int32_t* status;    // device status word
+  int sm_count;
+  std::string err;
+};
+
+// First device-side error wins.
+__device__ __forceinline__ void rc_set_status(int32_t* status, int32_t code) {
+  atomicCAS(status, 0, code);
+}
+
+// Largest i with cu[i] <= x, for cu[0..n] non-decreasing (n >= 1).
+__device__ __forceinline__ int rc_find_segment(const int32_t* __restrict__ cu, int n, int x) {
+  int lo = 0, hi = n;  // answer in [lo, hi)
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+template <typename T> __device__ __forceinline__ float rc_to_float(T x);
+template <> __device__ __forceinline__ float rc_to_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ float rc_to_float<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T rc_from_float(float x);
+template <> __device__ __forceinline__ float rc_from_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 rc_from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// ---- launchers (one per translation unit) -------------------------------
+// All return the cudaError_t of the launch (cudaGetLastError).
+
+// Rotates keys at their positions and stores keys/values head-major.
+//  mode 0 (encode): token t of resource i -> position t - cu[i], row slot[i] + (t - cu[i])
+//  mode 1 (prefill): token t of request b -> position pos0[b] + (t - cu[b]), row t
+struct RopeStoreArgs {
+  const void* k; const void* v;       // [total][G][d]
+  void* k_dst; void* v_dst;           // [G][dst_rows][d]
+  const int32_t* cu; int n_seq; int total;
+  const int32_t* slot;                // mode 0
+  const int32_t* pos0;                // mode 1
+  int64_t dst_rows;
+  int mode;
+};
+cudaError_t rc_launch_rope_store(const recache_ctx* ctx, const RopeStoreArgs& a, cudaStream_t st);
+
+// Generic row-per-warp attention (exact fp32 arithmetic; the fp32 path and the
+// small-shape path of bf16).
+struct AttnRowsArgs {
+  const void* q; void* o; int out_dtype;   // [total][Hq][d]
+  const int32_t* cu; int n_seq; int total; // sequences (resources or requests)
+  const int32_t* pos0;                     // null: positions start at 0
+  const int32_t* slot;                     // causal segment base row per sequence; null: cu[b]
+  const void* k_self; const void* v_self;  // [G][self_rows][d] rotated keys / values
+  int64_t self_rows;
+  const void* k_route; const void* v_route; const int32_t* route_cu;  // null for encode
+};
+cudaError_t rc_launch_attn_rows(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t st);
+
+struct CompactArgs {
+  const void* k_cache; const void* v_cache; int64_t pool_tokens;
+  const uint8_t* keep;
+  const int32_t* res_off; const int32_t* res_slot; const int32_t* res_len;
+  int n_requests; int total_listed;
+  const uint8_t* vis; int mode;
+  int32_t* route_cu; int32_t* route_len; int32_t* route_idx; int64_t row_capacity;
+  void* k_out; void* v_out;
+  int32_t* page_table; int max_pages_per_route;
+  const int32_t* free_pages; int64_t n_free_pages; int64_t n_pool_pages;
+  void* workspace;
+};
+int64_t rc_compact_workspace_bytes(const recache_ctx* ctx, int n_requests, int total_listed);
+cudaError_t rc_launch_compact(const recache_ctx* ctx, const CompactArgs& a, cudaStream_t st);
+
+struct DecodeArgs {
+  const void* q; const int32_t* q_pos; int batch;
+  const void* k_new; const void* v_new;
+  void* k_pages; void* v_pages; int64_t n_pages;
+  const int32_t* res_pt; int max_res_pages; const int32_t* res_len;
+  const int32_t* hist_pt; int max_hist_pages; const int32_t* hist_len;
+  void* o; int out_dtype;
+  void* workspace; int64_t workspace_bytes;
+};
+cudaError_t rc_launch_decode_append(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
+cudaError_t rc_launch_decode_rows(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
+
+// ---- dispatch between the exact-fp32 kernels and the bf16 tensor-core ones ----
+struct EncodeArgs {
+  const void* q; void* o; int out_dtype;
+  const int32_t* cu; int n_res; int total; int max_len;
+  const int32_t* slot; const void* k_cache; const void* v_cache; int64_t pool_tokens;
+  void* workspace; int64_t workspace_bytes;
+};
+struct PrefillArgs {
+  const void* q; void* o; int out_dtype;
+  const int32_t* cu_q; const int32_t* pos0; int n_req; int total_q; int max_q;
+  const void* k_route; const void* v_route; const int32_t* route_cu; int64_t route_rows;
+  const void* k_conv; const void* v_conv;   // rotated, [G][total_q][d]
+  void* workspace; int64_t workspace_bytes;
+};
+int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, int max_len);
+int64_t rc_prefill_workspace_bytes(const recache_ctx* ctx, int n_req, int total_q, int max_q);
+int64_t rc_decode_workspace_bytes(const recache_ctx* ctx, int batch, int max_res_pages, int max_hist_pages);
+cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, cudaStream_t st);
+cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a, cudaStream_t st);
+cudaError_t rc_launch_decode(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
