@@ -22,7 +22,10 @@ What follows which passage of the paper ("Section ReCache"):
 Readings taken where the paper is silent (all parameters here, none hidden):
 positions start at 0; RoPE pairs element i with i + d/2; scale 1/sqrt(d);
 query head h reads KV group h // (Hq/G); a route's rows are ordered by request
-order then ascending token; the cache stores rotated keys in the storage dtype.
+order then ascending token; rotated queries and keys are materialised in the
+storage dtype (`storage`: "bf16", "f32" or None = keep fp64) before the score
+product, as a transformer running in that dtype does, so the key a resource's
+own tokens attend to is the very key the cache holds for every later reader.
 
 Pins (tests/test_oracle_*.py): hand-computed RoPE values, brute-force masked
 attention in pure Python, torch's fp64 scaled_dot_product_attention on the
@@ -103,8 +106,8 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
         if n == 0:
             continue
         pos = np.arange(n) + (0 if pos_offset is None else int(pos_offset[i]))
-        qh = rope(q[a:b], pos, theta)
-        kh = rope(k[a:b], pos, theta)
+        qh = round_storage(rope(q[a:b], pos, theta), storage)
+        kh = round_storage(rope(k[a:b], pos, theta), storage)
         k_hat[a:b] = kh
         causal = np.tril(np.ones((n, n), dtype=bool))
         for h in range(hq):
@@ -112,10 +115,11 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
             sc = qh[:, h, :] @ kh[:, kg, :].T / math.sqrt(d)
             sc = np.where(causal, sc, -np.inf)
             o[a:b, h, :] = _softmax_rows(sc) @ v[a:b, kg, :]
-    return o, round_storage(k_hat, storage), v.copy()
+    return o, k_hat, v.copy()
 
 
-def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int]]):
+def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int]],
+                storage: Optional[str] = None):
     """The same definition for a chosen set of output rows (token, head) only,
     one at a time; for sizes where the full table takes minutes."""
     q = np.asarray(q, F64)
@@ -129,8 +133,8 @@ def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int
         a = int(cu[i])
         j = tok - a
         kg = h // s
-        qh = rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([j]), theta)[0, 0]
-        kh = rope(np.asarray(k[a:tok + 1, kg:kg + 1], F64), np.arange(j + 1), theta)[:, 0, :]
+        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([j]), theta), storage)[0, 0]
+        kh = round_storage(rope(np.asarray(k[a:tok + 1, kg:kg + 1], F64), np.arange(j + 1), theta), storage)[:, 0, :]
         sc = kh @ qh / math.sqrt(d)
         out[n] = _softmax_rows(sc[None, :])[0] @ np.asarray(v[a:tok + 1, kg, :], F64)
     return out
@@ -230,8 +234,8 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
         if n == 0:
             continue
         pos = int(q_pos0[b]) + np.arange(n)
-        qh = rope(q[a:e], pos, theta)
-        kh = rope(k_conv[a:e], pos, theta)
+        qh = round_storage(rope(q[a:e], pos, theta), storage)
+        kh = round_storage(rope(k_conv[a:e], pos, theta), storage)
         kc_hat[a:e] = kh
         causal = np.tril(np.ones((n, n), dtype=bool))
         for h in range(hq):
@@ -243,11 +247,11 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
             s_conv = np.where(causal, qh[:, h, :] @ kh[:, kg, :].T / math.sqrt(d), -np.inf)
             p = _softmax_rows(np.concatenate([s_res, s_conv], axis=1))
             o[a:e, h, :] = p @ np.concatenate([vr, v_conv[a:e, kg, :]], axis=0)
-    return o, round_storage(kc_hat, storage)
+    return o, kc_hat
 
 
 def prefill_rows(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta: float,
-                 out_rows: Sequence[Tuple[int, int]]):
+                 out_rows: Sequence[Tuple[int, int]], storage: Optional[str] = None):
     """attend_prefill for chosen (query token, head) rows only."""
     q = np.asarray(q); cu = np.asarray(cu_q)
     tq, hq, d = q.shape
@@ -260,8 +264,9 @@ def prefill_rows(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta:
         t = tok - a
         kg = h // s
         p0 = int(q_pos0[b])
-        qh = rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([p0 + t]), theta)[0, 0]
-        kh = rope(np.asarray(k_conv[a:tok + 1, kg:kg + 1], F64), p0 + np.arange(t + 1), theta)[:, 0, :]
+        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([p0 + t]), theta), storage)[0, 0]
+        kh = round_storage(rope(np.asarray(k_conv[a:tok + 1, kg:kg + 1], F64), p0 + np.arange(t + 1), theta),
+                           storage)[:, 0, :]
         r = rows[b][kg]
         keys = np.concatenate([np.asarray(k_cache[kg][r], F64).reshape(len(r), d), kh], axis=0)
         vals = np.concatenate([np.asarray(v_cache[kg][r], F64).reshape(len(r), d),
@@ -286,7 +291,8 @@ def append_decode_kv(k_pages, v_pages, hist_page_table, hist_len, k_new, v_new, 
 
 
 def attend_decode(q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page_table,
-                  hist_len, theta: float, page_tokens: int, items: Optional[Sequence[int]] = None):
+                  hist_len, theta: float, page_tokens: int, items: Optional[Sequence[int]] = None,
+                  storage: Optional[str] = None):
     """One query token per sequence over its route's paged resource rows and its
     paged history (whose last row is the current token).  q: [B,Hq,d] pre-RoPE.
     `items` restricts the work to chosen (sequence*G + group) items; other
@@ -295,7 +301,7 @@ def attend_decode(q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page
     b, hq, d = q.shape
     g = len(res_len) // b
     s = hq // g
-    qh = rope(q, np.asarray(q_pos), theta)
+    qh = round_storage(rope(q, np.asarray(q_pos), theta), storage)
     o = np.zeros_like(q)
 
     def rows_of(table, n):

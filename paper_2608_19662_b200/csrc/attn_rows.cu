@@ -67,14 +67,15 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
   if (pos < 0 || pos >= max_pos) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_POS); return; }
   if (base < 0 || base + j >= self_rows) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_SLOT); return; }
 
-  // rotate the query row into shared memory (fp32), folding in the softmax scale
+  // rotate the query row into shared memory
   constexpr int HALF = D / 2;
   const T* qrow = q + ((int64_t)t * Hq + h) * D;
   for (int i = lane; i < HALF; i += 32) {
     const float lo = rc_to_float<T>(qrow[i]), hi = rc_to_float<T>(qrow[i + HALF]);
     const float c = cos_tab[(int64_t)pos * HALF + i], s = sin_tab[(int64_t)pos * HALF + i];
-    q_s[warp][i] = __fmaf_rn(lo, c, -__fmul_rn(hi, s));
-    q_s[warp][i + HALF] = __fmaf_rn(hi, c, __fmul_rn(lo, s));
+    // the rotated query is a tensor of the storage dtype, like the cached keys
+    q_s[warp][i] = rc_to_float<T>(rc_from_float<T>(__fmaf_rn(lo, c, -__fmul_rn(hi, s))));
+    q_s[warp][i + HALF] = rc_to_float<T>(rc_from_float<T>(__fmaf_rn(hi, c, __fmul_rn(lo, s))));
   }
   __syncwarp();
 

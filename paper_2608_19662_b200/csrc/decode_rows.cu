@@ -59,8 +59,9 @@ __global__ void __launch_bounds__(WARPS * 32) decode_rows_kernel(
   for (int i = lane; i < HALF; i += 32) {
     const float lo = rc_to_float<T>(qrow[i]), hi = rc_to_float<T>(qrow[i + HALF]);
     const float c = cos_tab[(int64_t)pos * HALF + i], s = sin_tab[(int64_t)pos * HALF + i];
-    q_s[warp][i] = __fmaf_rn(lo, c, -__fmul_rn(hi, s));
-    q_s[warp][i + HALF] = __fmaf_rn(hi, c, __fmul_rn(lo, s));
+    // the rotated query is a tensor of the storage dtype, like the cached keys
+    q_s[warp][i] = rc_to_float<T>(rc_from_float<T>(__fmaf_rn(lo, c, -__fmul_rn(hi, s))));
+    q_s[warp][i + HALF] = rc_to_float<T>(rc_from_float<T>(__fmaf_rn(hi, c, __fmul_rn(lo, s))));
   }
   __syncwarp();
   constexpr int CPL = D / 32;

@@ -29,12 +29,21 @@ def check_cache(shape, kc_gpu, vc_gpu, kc_ref, vc_ref):
     written = ~np.isnan(kc_ref)
     assert np.array_equal(np.isnan(f64(kc_gpu)), ~written)       # only the resources' rows are written
     assert np.array_equal(f64(vc_gpu)[written], vc_ref[written])
+    assert_rotated_close(shape, kc_gpu, np.where(written, kc_ref, 0.0), written)
+
+
+def assert_rotated_close(shape, got, ref, mask=None):
+    """fp32 rotation on the GPU against the fp64 one: equal up to one unit in the
+    last place of the storage type (plus the fp32 rounding of the two products,
+    which matters only where they cancel), and different in few places."""
+    mask = np.ones(ref.shape, bool) if mask is None else mask
+    diff = np.abs(f64(got) - ref)[mask]
     if shape.dtype == "bf16":
-        ulps = bf16_ulp_distance(kc_gpu, np.where(written, kc_ref, 0.0))[written]
-        assert ulps.max() <= 1.0
-        assert (ulps > 0).mean() < 0.01
+        ulps = bf16_ulp_distance(got, ref)[mask]
+        assert ((ulps <= 1.0) | (diff < 2e-6)).all()
+        assert (diff > 0).mean() < 0.01
     else:
-        assert np.abs(f64(kc_gpu)[written] - kc_ref[written]).max() < 2e-6
+        assert diff.max() < 2e-6
 
 
 def check_compaction(out, rows, kc_gpu, vc_gpu, shape):
@@ -84,7 +93,7 @@ def test_config1_fp32_whole_path():
     p_ref, kconv_ref = oracle_prefill(req, rows, kc_ref, vc_ref)
     p, kconv, vconv = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
     assert max_abs(p, p_ref) < TOL_F32
-    assert max_abs(kconv, np.transpose(kconv_ref, (1, 0, 2))) < 2e-6
+    assert_rotated_close(sh, kconv, np.transpose(kconv_ref, (1, 0, 2)))
     assert torch.equal(vconv.cpu(), req.v_conv.permute(1, 0, 2))
     assert_status_ok(rc)
 
@@ -138,7 +147,7 @@ def test_config1_decode_equals_last_prefill_row():
                          sh.rope_theta, pt, storage=sh.dtype)
     res_len = np.array([len(r) for r in rows[0]], np.int32)
     od_ref = orc.attend_decode(f64(req.q)[tq - 1:tq], q_pos, kp_ref, vp_ref, table_ref, res_len, hist_pt, hist_len,
-                               sh.rope_theta, pt)
+                               sh.rope_theta, pt, storage=sh.dtype)
     assert max_abs(od, od_ref) < TOL_F32
     assert max_abs(od, p_ref[tq - 1:tq]) < TOL_F32
     assert_status_ok(rc)
@@ -164,7 +173,7 @@ def test_config2_bf16_whole_path(out_dtype):
     p_ref, kconv_ref = oracle_prefill(req, rows, kc_ref, vc_ref)
     p, kconv, vconv = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"], out_dtype=out_dtype)
     assert (np.abs(f64(p) - p_ref) <= TOL_BF16 + slack * np.abs(p_ref)).all()
-    assert bf16_ulp_distance(kconv, np.transpose(kconv_ref, (1, 0, 2))).max() <= 1.0
+    assert_rotated_close(sh, kconv, np.transpose(kconv_ref, (1, 0, 2)))
     assert torch.equal(vconv.cpu(), req.v_conv.permute(1, 0, 2))
     assert_status_ok(rc)
 
@@ -224,7 +233,8 @@ def test_config4_decode_small_batch():
     od = rc.attend_decode(dev(dec.q), dev(dec.q_pos), dev(dec.k_pages), dev(dec.v_pages), dev(dec.res_page_table),
                           dev(dec.res_len), dev(dec.hist_page_table), dev(dec.hist_len), out_dtype=torch.float32)
     ref = orc.attend_decode(f64(dec.q), dec.q_pos, f64(dec.k_pages), f64(dec.v_pages), dec.res_page_table,
-                            dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS)
+                            dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS,
+                            storage=sh.dtype)
     assert max_abs(od, ref) < TOL_BF16
     assert_status_ok(rc)
 
@@ -238,7 +248,8 @@ def test_config4_decode_full_size_sampled_items():
                           dev(dec.res_len), dev(dec.hist_page_table), dev(dec.hist_len), out_dtype=torch.float32)
     items = sorted(set([0, 511] + [int(x) for x in np.random.default_rng(4).integers(0, 512, 30)]))
     ref = orc.attend_decode(f64(dec.q), dec.q_pos, dec.k_pages, dec.v_pages, dec.res_page_table,
-                            dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS, items=items)
+                            dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS, items=items,
+                            storage=sh.dtype)
     g, s = sh.n_kv_heads, sh.group_size
     for it in items:
         b, kg = divmod(it, g)
