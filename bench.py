@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the resource-routed attention hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+  1. recache_encode_resources   long-tool-set: 64 resources U[1000,2000] tokens
+  2. recache_compact_routes     packed, 25 % routes x ~30 % kept tokens
+  3. recache_attend_prefill     2048 conversation tokens over the routed KV
+  4. recache_compact_routes     paged, for a 64-sequence decode batch
+  5. recache_attend_decode      64 x 1 token over ~720 resource rows + 2048 history rows
+(workloads 5 and 4 of the build: Qwen3-class shape, 32 query / 8 KV heads,
+head_dim 128, bf16 storage with fp32 accumulation).
+
+value   = useful attention TFLOP/s over the whole step (4*d FLOP per unmasked
+          (query, key) pair, masked or padded tile area never counted), inputs
+          resident in HBM.
+e2e     = the same with every step's inputs copied from pinned host memory and
+          its outputs copied back inside the timed region.
+roofline= dominant kernel (the encode attention) against the measured bf16 peak;
+          `stages` also reports decode and compaction against measured HBM bandwidth.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--small]
+Under torchrun every rank runs an independent replica (the path has no exchange
+step); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_19662_b200 import workloads as wl  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ workload --
+class Workload:
+    """Host-side (pinned) inputs + the algorithmic work they amount to."""
+
+    def __init__(self, small: bool, seed_shift: int = 0):
+        sh = wl.QWEN3_4B
+        self.shape = sh
+        if small:
+            self.pool, self.req = wl.config5(n_res=6, len_range=(300, 700), tq=256, seed=wl.SEED0 + 5 + seed_shift)
+            self.dc = wl.config4_compose(batch=4, n_res=8, res_len=(100, 260), hist=300, seed=wl.SEED0 + 4 + seed_shift)
+            self.name = "small: 6 resources U[300,700] + 256-token prefill; decode batch 4"
+        else:
+            self.pool, self.req = wl.config5(seed=wl.SEED0 + 5 + seed_shift)
+            self.dc = wl.config4_compose(seed=wl.SEED0 + 4 + seed_shift)
+            self.name = ("long-tool-set (64 resources U[1000,2000], 2048-token prefill, 25% routes x 30% kept) "
+                         "+ routed decode (batch 64, 16 resources ~600 tok, 2048 history, 64-token pages)")
+        d, hq, g = sh.head_dim, sh.n_q_heads, sh.n_kv_heads
+        dc = self.dc
+        self.dec_q = wl.normal(901 + seed_shift, (dc.batch, hq, d), sh.torch_dtype)
+        self.dec_k_new = wl.normal(902 + seed_shift, (dc.batch, g, d), sh.torch_dtype)
+        self.dec_v_new = wl.normal(903 + seed_shift, (dc.batch, g, d), sh.torch_dtype)
+        self.max_pos = int(max(self.req.q_pos0.max() + self.req.max_q, dc.q_pos.max() + 1, self.pool.max_len)) + 1
+
+        # algorithmic work
+        lens = self.pool.lens.astype(np.int64)
+        self.pairs_encode = int((lens * (lens + 1) // 2).sum()) * hq
+        kept = np.array([int(self.pool.keep[s:s + n].sum()) for s, n in zip(self.pool.dst_slot, self.pool.lens)])
+        self.route_len = (self.req.vis.astype(np.int64) * kept[None, :]).sum(1)          # [G], one request
+        tq = self.req.total_q
+        self.pairs_prefill = int(sum(sh.group_size * (tq * int(n) + tq * (tq + 1) // 2) for n in self.route_len))
+        kept4 = np.add.reduceat(dc.keep.astype(np.int64), dc.dst_slot)
+        n_res = len(dc.lens) // dc.batch
+        rl4 = np.array([[int((dc.vis[kg, b * n_res:(b + 1) * n_res] * kept4[b * n_res:(b + 1) * n_res]).sum())
+                         for kg in range(g)] for b in range(dc.batch)]).reshape(-1)
+        self.dec_rows = int(rl4.sum() + dc.hist_len.sum())
+        self.pairs_decode = self.dec_rows * sh.group_size
+        self.flops = {k: 4 * d * v for k, v in (("encode", self.pairs_encode), ("prefill", self.pairs_prefill),
+                                                ("decode", self.pairs_decode))}
+        row_b = d * 2
+        self.bytes = {
+            "decode": self.dec_rows * 2 * row_b,
+            "compact_packed": int(self.route_len.sum()) * (4 * row_b + 4),
+            "compact_paged": int(rl4.sum()) * (4 * row_b + 4),
+            "rope_store": (self.pool.total_tokens + tq) * g * 4 * row_b,
+        }
+        self.total_flops = sum(self.flops.values())
+
+    def host_inputs(self):
+        """Everything a step consumes, as pinned host tensors."""
+        p, r, dc = self.pool, self.req, self.dc
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a))
+        h = dict(q=p.q, k=p.k, v=p.v, cu=t(p.cu_seqlens), slot=t(p.dst_slot), keep=t(p.keep),
+                 res_off=t(r.res_off), res_slot=t(r.res_slot), res_len=t(r.res_len), vis=t(r.vis),
+                 cq=r.q, ck=r.k_conv, cv=r.v_conv, cu_q=t(r.cu_q), q_pos0=t(r.q_pos0),
+                 d_keep=t(dc.keep), d_res_off=t(dc.res_off), d_res_slot=t(dc.dst_slot), d_res_len=t(dc.lens),
+                 d_vis=t(dc.vis), d_free=t(dc.free_pages), d_hist_pt=t(dc.hist_page_table),
+                 d_hist_len=t(dc.hist_len), d_q=self.dec_q, d_kn=self.dec_k_new, d_vn=self.dec_v_new,
+                 d_q_pos=t(dc.q_pos))
+        return {k: v.contiguous().pin_memory() for k, v in h.items()}
+
+
+class Runner:
+    """Device state + one step of the hot path through the binding."""
+
+    def __init__(self, w: Workload, device: int):
+        from paper_2608_19662_b200 import ReCache
+        self.w = w
+        sh = w.shape
+        self.dev = torch.device("cuda", device)
+        self.rc = ReCache(sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.rope_theta, sh.dtype, max_pos=w.max_pos,
+                          page_tokens=wl.PAGE_TOKENS, device=device)
+        self.host = w.host_inputs()
+        self.d = {k: v.to(self.dev, non_blocking=True) for k, v in self.host.items()}
+        g, d, dt = sh.n_kv_heads, sh.head_dim, sh.torch_dtype
+        p, r, dc = w.pool, w.req, w.dc
+        E = lambda *s, dtype=dt: torch.empty(s, dtype=dtype, device=self.dev)
+        self.k_cache, self.v_cache = E(g, p.pool_tokens, d), E(g, p.pool_tokens, d)
+        self.o_enc = E(p.total_tokens, sh.n_q_heads, d)
+        cap = int(w.route_len.sum()) + 64
+        self.route_cu = E(g + 1, dtype=torch.int32)
+        self.route_idx = E(cap, dtype=torch.int32)
+        self.k_route, self.v_route = E(cap, d), E(cap, d)
+        self.o_pre = E(r.total_q, sh.n_q_heads, d)
+        self.k_conv_out, self.v_conv_out = E(g, r.total_q, d), E(g, r.total_q, d)
+        # decode state: a resident cache pool (stand-in for earlier encodes) and the page pool
+        self.d_k_cache = wl.seeded_normal(77, (g, dc.pool_tokens, d), dt, device=self.dev)
+        self.d_v_cache = wl.seeded_normal(78, (g, dc.pool_tokens, d), dt, device=self.dev)
+        self.k_pages = wl.seeded_normal(79, (dc.n_pages, wl.PAGE_TOKENS, d), dt, device=self.dev)
+        self.v_pages = wl.seeded_normal(80, (dc.n_pages, wl.PAGE_TOKENS, d), dt, device=self.dev)
+        n_items = dc.batch * g
+        self.d_route_cu = E(n_items + 1, dtype=torch.int32)
+        self.d_route_len = E(n_items, dtype=torch.int32)
+        self.d_route_idx = E(int(dc.keep.sum()) * 1 + 64, dtype=torch.int32)
+        self.d_page_table = E(n_items, dc.max_res_pages, dtype=torch.int32)
+        self.o_dec = E(dc.batch, sh.n_q_heads, d)
+        rc = self.rc
+        ws = max(rc.encode_workspace_bytes(len(p.lens), p.total_tokens, p.max_len),
+                 rc.compact_workspace_bytes(1, len(r.res_slot)), rc.prefill_workspace_bytes(1, r.total_q, r.max_q),
+                 rc.compact_workspace_bytes(dc.batch, len(dc.lens)),
+                 rc.decode_workspace_bytes(dc.batch, dc.max_res_pages, dc.hist_page_table.shape[1]), 256)
+        self.ws = torch.empty(ws, dtype=torch.uint8, device=self.dev)
+        # host landing buffers for the end-to-end variant
+        self.h_o_enc = torch.empty(self.o_enc.shape, dtype=dt).pin_memory()
+        self.h_o_pre = torch.empty(self.o_pre.shape, dtype=dt).pin_memory()
+        self.h_o_dec = torch.empty(self.o_dec.shape, dtype=dt).pin_memory()
+        self.h2d_bytes = sum(v.numel() * v.element_size() for v in self.host.values())
+        self.d2h_bytes = sum(v.numel() * v.element_size() for v in (self.h_o_enc, self.h_o_pre, self.h_o_dec))
+        torch.cuda.synchronize(self.dev)
+
+    def step(self):
+        from paper_2608_19662_b200 import PACKED, PAGED
+        rc, d, w = self.rc, self.d, self.w
+        p, r = w.pool, w.req
+        rc.encode_resources(d["q"], d["k"], d["v"], d["cu"], p.max_len, d["slot"], self.k_cache, self.v_cache,
+                            out=self.o_enc, workspace=self.ws)
+        rc.compact_routes(self.k_cache, self.v_cache, d["keep"], d["res_off"], d["res_slot"], d["res_len"], d["vis"],
+                          PACKED, self.route_cu, self.route_idx, self.k_route, self.v_route, workspace=self.ws)
+        rc.attend_prefill(d["cq"], d["ck"], d["cv"], d["cu_q"], d["q_pos0"], r.max_q, self.k_route, self.v_route,
+                          self.route_cu, k_conv_out=self.k_conv_out, v_conv_out=self.v_conv_out, out=self.o_pre,
+                          workspace=self.ws)
+        rc.compact_routes(self.d_k_cache, self.d_v_cache, d["d_keep"], d["d_res_off"], d["d_res_slot"], d["d_res_len"],
+                          d["d_vis"], PAGED, self.d_route_cu, self.d_route_idx, self.k_pages, self.v_pages,
+                          route_len=self.d_route_len, page_table=self.d_page_table, free_pages=d["d_free"],
+                          workspace=self.ws)
+        rc.attend_decode(d["d_q"], d["d_q_pos"], self.k_pages, self.v_pages, self.d_page_table, self.d_route_len,
+                         d["d_hist_pt"], d["d_hist_len"], k_new=d["d_kn"], v_new=d["d_vn"], out=self.o_dec,
+                         workspace=self.ws)
+
+    def step_e2e(self):
+        for k, v in self.host.items():
+            self.d[k].copy_(v, non_blocking=True)
+        self.step()
+        self.h_o_enc.copy_(self.o_enc, non_blocking=True)
+        self.h_o_pre.copy_(self.o_pre, non_blocking=True)
+        self.h_o_dec.copy_(self.o_dec, non_blocking=True)
+
+
+# --------------------------------------------------------------------- clocks --
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            out, _ = self.p.communicate(timeout=5)
+        except Exception:
+            self.p.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------- oracle sample --
+def oracle_sample(w: Workload, budget: str = "default"):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the same
+    workload: whole resources for a few heads (encode), a block of query tokens
+    (prefill) and a few decode items.  Returns (flops, seconds, description)."""
+    from oracle import recache_oracle as orc
+    sh = w.shape
+    p, r, dc = w.pool, w.req, w.dc
+    d, s = sh.head_dim, sh.group_size
+    f64 = lambda t: t.to(torch.float64).numpy()
+    n_res = min(12, len(p.lens))
+    ng = min(2, sh.n_kv_heads)
+    t_end = int(p.cu_seqlens[n_res])
+    t0 = time.perf_counter()
+    # encode: first n_res resources, query heads of the first ng KV groups
+    orc.encode_resources(f64(p.q[:t_end, :ng * s]), f64(p.k[:t_end, :ng]), f64(p.v[:t_end, :ng]),
+                         p.cu_seqlens[:n_res + 1], sh.rope_theta, storage=sh.dtype)
+    lens = p.lens[:n_res].astype(np.int64)
+    flops = 4 * d * ng * s * int((lens * (lens + 1) // 2).sum())
+    # prefill: first 128 query tokens, group 0, against that group's routed rows
+    rows = orc.compact_routes(p.keep, r.res_off, r.res_slot, r.res_len, r.vis[:1])
+    kc = np.zeros((1, p.pool_tokens, d)); vc = np.zeros_like(kc)
+    rng = np.random.default_rng(0)
+    kc[0, rows[0][0]] = rng.standard_normal((len(rows[0][0]), d)); vc[0, rows[0][0]] = 1.0
+    tq = min(512, r.total_q)
+    orc.attend_prefill(f64(r.q[:tq, :s]), f64(r.k_conv[:tq, :1]), f64(r.v_conv[:tq, :1]), [0, tq], r.q_pos0, rows,
+                       kc, vc, sh.rope_theta, storage=sh.dtype)
+    flops += 4 * d * s * (tq * len(rows[0][0]) + tq * (tq + 1) // 2)
+    # decode: 8 items over synthetic pages of the workload's lengths
+    n_it = 32
+    hist = int(dc.hist_len[0]); res = 720 if hist >= 2048 else 200
+    pt = wl.PAGE_TOKENS
+    n_pg = n_it * ((hist + pt - 1) // pt + (res + pt - 1) // pt)
+    kp = rng.standard_normal((n_pg, pt, d)); vp = rng.standard_normal((n_pg, pt, d))
+    ids = np.arange(n_pg, dtype=np.int32).reshape(n_it, -1)
+    rp = (res + pt - 1) // pt
+    orc.attend_decode(rng.standard_normal((n_it, s, d)), np.full(n_it, 100), kp, vp, ids[:, :rp],
+                      np.full(n_it, res), ids[:, rp:], np.full(n_it, hist), sh.rope_theta, pt, storage=sh.dtype)
+    flops += 4 * d * s * n_it * (res + hist)
+    sec = time.perf_counter() - t0
+    what = (f"encode of the first {n_res} resources ({t_end} tokens) for the {ng * s} query heads of {ng} KV groups + "
+            f"prefill of {tq} query tokens on one route + decode of {n_it} (sequence, group) items")
+    return flops, sec, what
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is the bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = Workload(args.small)
+    for _ in range(args.warmup):
+        oracle_sample(w)
+    t0 = time.perf_counter(); fl = 0
+    for _ in range(args.steps):
+        f, _, what = oracle_sample(w)
+        fl += f
+    sec = time.perf_counter() - t0
+    val = fl / sec / 1e12
+    cores = torch.get_num_threads()
+    line = {"impl": "reference", "metric": "routed_attn_useful_tflops", "value": val, "unit": "TFLOP/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sample": what},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------ main --
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--small", action="store_true", help="a small case (for profiler captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if dist:
+        import torch.distributed as td
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        td.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local)
+    peaks, peak_src = load_peaks()
+
+    w = Workload(args.small, seed_shift=rank)
+    run = Runner(w, local)
+    rc = run.rc
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, with_timer=False):
+        for _ in range(max(args.warmup, 3) if not args.small else args.warmup):
+            fn()
+        barrier()
+        if with_timer:
+            rc.kernel_timer(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler = ClockSampler(local) if with_timer else None
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop() if sampler else None
+        kt = rc.kernel_times() if with_timer else None
+        if with_timer:
+            rc.kernel_timer(False)
+        if dist:
+            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            td.all_reduce(t, op=td.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, kt, clocks
+
+    ms, kt, clocks = timed(run.step, args.steps, with_timer=True)
+    code = rc.poll_status()
+    if code != 0:
+        raise SystemExit(f"device status {code} after the timed region")
+    ms_step = ms / args.steps
+    value = world * w.total_flops / (ms_step * 1e-3) / 1e12
+
+    e2e = None
+    if not args.no_e2e:
+        ms_e, _, _ = timed(run.step_e2e, args.steps)
+        e2e = {"value": world * w.total_flops / (ms_e / args.steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "ms_per_step": ms_e / args.steps, "h2d_bytes_per_step": run.h2d_bytes,
+               "d2h_bytes_per_step": run.d2h_bytes}
+
+    # per-kernel accounting from the library's event pairs
+    per = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in kt.items() if v[1]}
+    launches = int(sum(v[1] for v in kt.values()))
+    enc_ms = kt["encode_attn"][0] / max(kt["encode_attn"][1], 1)
+    ach = w.flops["encode"] / (enc_ms * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roofline = {"kernel": "encode_attn", "bound": "tensor", "achieved": ach, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": ach / peak_tf, "traffic": None, "peak_source": f"{peak_src} (sustained bf16)",
+                "flops_per_launch": w.flops["encode"], "ms_per_launch": enc_ms}
+    stages = {}
+    if "prefill_attn" in per:
+        t = per["prefill_attn"]["ms_per_step"]
+        stages["prefill_attn"] = {"tflops": w.flops["prefill"] / (t * 1e-3) / 1e12, "ms": t,
+                                  "frac_of_bf16_peak": w.flops["prefill"] / (t * 1e-3) / 1e12 / peak_tf}
+    if "decode_attn" in per:
+        t = per["decode_attn"]["ms_per_step"] + per.get("decode_merge", {"ms_per_step": 0})["ms_per_step"]
+        gbs = w.bytes["decode"] / (t * 1e-3) / 1e9
+        stages["decode_attn"] = {"gbs": gbs, "ms": t, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                                 "bytes": w.bytes["decode"]}
+    if "compact_gather" in per:
+        t = per["compact_gather"]["ms_per_step"]
+        b = w.bytes["compact_packed"] + w.bytes["compact_paged"]
+        stages["compact_gather"] = {"gbs": b / (t * 1e-3) / 1e9, "ms": t, "frac_of_hbm_peak": b / (t * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    if "rope_store" in per:
+        t = per["rope_store"]["ms_per_step"]
+        stages["rope_store"] = {"gbs": w.bytes["rope_store"] / (t * 1e-3) / 1e9, "ms": t,
+                                "frac_of_hbm_peak": w.bytes["rope_store"] / (t * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        f, sec, what = oracle_sample(w)
+        cpu = {"value": f / sec / 1e12, "unit": "TFLOP/s", "cores": torch.get_num_threads(), "kind": "oracle",
+               "sample": what, "seconds": sec}
+
+    if rank == 0:
+        line = {"metric": "routed_attn_useful_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3) if not args.small else args.warmup,
+                "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": w.name, "l2": "inputs larger than L2 (encode inputs ~1.2 GB per step)",
+                           "shape": "32 q heads / 8 kv heads / head_dim 128", "parallelism": f"replicas x{world}",
+                           "useful_tflop_per_step": w.total_flops / 1e12,
+                           "flops": {k: v / 1e12 for k, v in w.flops.items()}},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+                "cpu_baseline": cpu, "stages": stages, "kernels": per}
+        print(json.dumps(line))
+    if dist:
+        td.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

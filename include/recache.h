@@ -103,6 +103,23 @@ RECACHE_API const char* recache_last_error(const recache_ctx* ctx);
  * clears it. */
 RECACHE_API recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* device_code);
 
+/*
+ * Launch accounting.  The library counts every kernel it launches; with the
+ * timer enabled it also records a CUDA event pair around each launch on the
+ * launch stream (a few microseconds of host time per launch).
+ *   recache_kernel_count()      number of distinct kernels K
+ *   recache_kernel_name(id)     static string, id in [0, K)
+ *   recache_kernel_timer(ctx,e) enable (1) / disable (0); clears counters and pending events
+ *   recache_kernel_times(ctx, ms_total[K], launches[K])  waits for the recorded
+ *       events, returns per-kernel summed device time in ms (0 when the timer
+ *       was off) and launch counts since the last clear, then clears both.
+ * Host arrays; no paper counterpart (measurement aid).
+ */
+RECACHE_API int32_t recache_kernel_count(void);
+RECACHE_API const char* recache_kernel_name(int32_t id);
+RECACHE_API recache_status recache_kernel_timer(recache_ctx* ctx, int32_t enable);
+RECACHE_API recache_status recache_kernel_times(recache_ctx* ctx, float* ms_total, int64_t* launches);
+
 /* Scratch sizes in bytes for the calls below (same size arguments). */
 RECACHE_API int64_t recache_encode_workspace_bytes(const recache_ctx* ctx, int32_t n_resources,
                                        int32_t total_tokens, int32_t max_len);

@@ -35,6 +35,10 @@ SIGNATURES = {
     "recache_destroy": (None, [_P]),
     "recache_last_error": (C.c_char_p, [_P]),
     "recache_poll_status": (C.c_int, [_P, _P, C.POINTER(_I32)]),
+    "recache_kernel_count": (_I32, []),
+    "recache_kernel_name": (C.c_char_p, [_I32]),
+    "recache_kernel_timer": (C.c_int, [_P, _I32]),
+    "recache_kernel_times": (C.c_int, [_P, C.POINTER(C.c_float), C.POINTER(_I64)]),
     "recache_encode_workspace_bytes": (_I64, [_P, _I32, _I32, _I32]),
     "recache_compact_workspace_bytes": (_I64, [_P, _I32, _I32]),
     "recache_prefill_workspace_bytes": (_I64, [_P, _I32, _I32, _I32]),
@@ -133,6 +137,17 @@ class ReCache:
         code = _I32(0)
         self._check(self.lib.recache_poll_status(self.h, _stream(), C.byref(code)), "recache_poll_status")
         return int(code.value)
+
+    def kernel_timer(self, enable: bool):
+        self._check(self.lib.recache_kernel_timer(self.h, 1 if enable else 0), "recache_kernel_timer")
+
+    def kernel_times(self):
+        """{kernel name: (total ms, launches)} since the last call; clears the counters."""
+        n = self.lib.recache_kernel_count()
+        ms = (C.c_float * n)()
+        cnt = (_I64 * n)()
+        self._check(self.lib.recache_kernel_times(self.h, ms, cnt), "recache_kernel_times")
+        return {self.lib.recache_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     # -------------------------------------------------------------- hot path --
     def encode_workspace_bytes(self, n_resources, total_tokens, max_len) -> int:

@@ -21,6 +21,12 @@ bool out_dtype_ok(const recache_ctx* ctx, int out_dtype) {
 }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+void clear_timer(recache_ctx* ctx) {
+  for (auto& t : ctx->timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+  ctx->timed.clear();
+  for (int i = 0; i < RC_K_COUNT; ++i) ctx->launches[i] = 0;
+}
+
 #define RC_REQUIRE(cond, st, msg) do { if (!(cond)) return fail(ctx, st, msg); } while (0)
 #define RC_CUDA(expr, where) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return cuda_fail(ctx, e_, where); } while (0)
 
@@ -76,6 +82,7 @@ void recache_destroy(recache_ctx* ctx) {
   cudaFree(ctx->cos_tab);
   cudaFree(ctx->sin_tab);
   cudaFree(ctx->status);
+  clear_timer(ctx);
   delete ctx;
 }
 
@@ -89,6 +96,33 @@ recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* devi
   RC_CUDA(cudaMemsetAsync(ctx->status, 0, sizeof(int32_t), st), "poll clear");
   RC_CUDA(cudaStreamSynchronize(st), "poll sync");
   *device_code = code;
+  return RECACHE_OK;
+}
+
+static const char* kKernelNames[RC_K_COUNT] = {
+    "rope_store", "tile_plan", "encode_attn", "prefill_attn", "compact_count", "compact_plan",
+    "compact_gather", "decode_append", "decode_attn", "decode_merge"};
+
+int32_t recache_kernel_count(void) { return RC_K_COUNT; }
+const char* recache_kernel_name(int32_t id) { return (id >= 0 && id < RC_K_COUNT) ? kKernelNames[id] : ""; }
+
+recache_status recache_kernel_timer(recache_ctx* ctx, int32_t enable) {
+  if (!ctx) return RECACHE_EINVAL;
+  clear_timer(ctx);
+  ctx->timer_on = enable != 0;
+  return RECACHE_OK;
+}
+
+recache_status recache_kernel_times(recache_ctx* ctx, float* ms_total, int64_t* launches) {
+  if (!ctx || !ms_total || !launches) return RECACHE_EINVAL;
+  for (int i = 0; i < RC_K_COUNT; ++i) { ms_total[i] = 0.f; launches[i] = ctx->launches[i]; }
+  for (auto& t : ctx->timed) {
+    RC_CUDA(cudaEventSynchronize(t.stop), "kernel_times: event sync");
+    float ms = 0.f;
+    RC_CUDA(cudaEventElapsedTime(&ms, t.start, t.stop), "kernel_times: elapsed");
+    ms_total[t.id] += ms;
+  }
+  clear_timer(ctx);
   return RECACHE_OK;
 }
 

@@ -136,6 +136,7 @@ cudaError_t launch(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t s
   if (rows == 0) return cudaSuccess;
   const unsigned blocks = (unsigned)((rows + WARPS - 1) / WARPS);
   const float scale = (float)(1.0 / sqrt((double)d));
+  RcLaunchScope scope(ctx, a.route_cu ? RC_K_PREFILL_ATTN : RC_K_ENCODE_ATTN, st);
 #define RC_ARGS (const T*)a.q, (TO*)a.o, a.cu, a.n_seq, a.total, a.pos0, a.slot, (const T*)a.k_self, \
     (const T*)a.v_self, a.self_rows, (const T*)a.k_route, (const T*)a.v_route, a.route_cu, Hq, G,    \
     ctx->cos_tab, ctx->sin_tab, ctx->desc.max_pos, scale, ctx->status

@@ -4,8 +4,18 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <string>
+#include <vector>
 
 #include "recache.h"
+
+// Kernels of the library, for launch counting and optional per-kernel timing.
+enum RcKernel {
+  RC_K_ROPE_STORE = 0, RC_K_TILE_PLAN, RC_K_ENCODE_ATTN, RC_K_PREFILL_ATTN,
+  RC_K_COMPACT_COUNT, RC_K_COMPACT_PLAN, RC_K_COMPACT_GATHER,
+  RC_K_DECODE_APPEND, RC_K_DECODE_ATTN, RC_K_DECODE_MERGE, RC_K_COUNT
+};
+
+struct RcTimedLaunch { int id; cudaEvent_t start, stop; };
 
 struct recache_ctx {
   recache_desc desc;
@@ -15,6 +25,28 @@ struct recache_ctx {
   int32_t* status;    // device status word
   int sm_count;
   std::string err;
+  // launch accounting (host side only)
+  mutable bool timer_on = false;
+  mutable int64_t launches[RC_K_COUNT] = {0};
+  mutable std::vector<RcTimedLaunch> timed;
+};
+
+// Brackets one kernel launch: counts it, and when the timer is enabled records
+// a CUDA event pair around it on the launch stream.
+struct RcLaunchScope {
+  const recache_ctx* ctx; cudaStream_t st; cudaEvent_t stop = nullptr;
+  RcLaunchScope(const recache_ctx* c, int id, cudaStream_t s) : ctx(c), st(s) {
+    ctx->launches[id]++;
+    if (ctx->timer_on) {
+      RcTimedLaunch t{id, nullptr, nullptr};
+      if (cudaEventCreate(&t.start) == cudaSuccess && cudaEventCreate(&t.stop) == cudaSuccess) {
+        cudaEventRecord(t.start, st);
+        stop = t.stop;
+        ctx->timed.push_back(t);
+      }
+    }
+  }
+  ~RcLaunchScope() { if (stop) cudaEventRecord(stop, st); }
 };
 
 // First device-side error wins.

@@ -228,15 +228,20 @@ cudaError_t rc_launch_compact(const recache_ctx* ctx, const CompactArgs& a, cuda
   Ws w = carve(a.workspace, n_routes, a.total_listed, G);
   if (a.total_listed > 0) {
     const int blocks = a.total_listed < 4096 ? a.total_listed : 4096;
+    RcLaunchScope scope(ctx, RC_K_COMPACT_COUNT, st);
     compact_count_kernel<<<blocks, TPB, 0, st>>>(a.keep, a.res_slot, a.res_len, a.total_listed,
                                                  a.pool_tokens, w.kept, ctx->status);
   }
-  compact_plan_kernel<<<1, 1024, 0, st>>>(w.kept, a.res_off, a.n_requests, a.total_listed, a.vis, G, a.mode,
-                                          ctx->desc.page_tokens, a.route_cu, a.route_len, w.res_route_off,
-                                          w.page_cu, a.row_capacity, a.page_table, a.max_pages_per_route,
-                                          a.free_pages, a.n_free_pages, a.n_pool_pages, ctx->status);
+  {
+    RcLaunchScope scope(ctx, RC_K_COMPACT_PLAN, st);
+    compact_plan_kernel<<<1, 1024, 0, st>>>(w.kept, a.res_off, a.n_requests, a.total_listed, a.vis, G, a.mode,
+                                            ctx->desc.page_tokens, a.route_cu, a.route_len, w.res_route_off,
+                                            w.page_cu, a.row_capacity, a.page_table, a.max_pages_per_route,
+                                            a.free_pages, a.n_free_pages, a.n_pool_pages, ctx->status);
+  }
   if (a.total_listed > 0) {
     dim3 grid((unsigned)a.total_listed, (unsigned)G);
+    RcLaunchScope scope(ctx, RC_K_COMPACT_GATHER, st);
     compact_gather_kernel<<<grid, TPB, 0, st>>>(
         (const uint8_t*)a.k_cache, (const uint8_t*)a.v_cache, a.pool_tokens, a.keep, a.res_off, a.res_slot,
         a.res_len, a.n_requests, a.total_listed, a.vis, G, a.mode, ctx->desc.page_tokens, a.route_cu,

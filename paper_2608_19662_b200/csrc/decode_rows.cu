@@ -126,6 +126,7 @@ cudaError_t launch_rows(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_
   const int rows = a.batch * Hq;
   const unsigned blocks = (unsigned)((rows + WARPS - 1) / WARPS);
   const float scale = (float)(1.0 / sqrt((double)d));
+  RcLaunchScope scope(ctx, RC_K_DECODE_ATTN, st);
 #define RC_ARGS (const T*)a.q, a.q_pos, a.batch, (const T*)a.k_pages, (const T*)a.v_pages, a.n_pages, a.res_pt, \
     a.max_res_pages, a.res_len, a.hist_pt, a.max_hist_pages, a.hist_len, (TO*)a.o, Hq, G,                       \
     ctx->desc.page_tokens, ctx->cos_tab, ctx->sin_tab, ctx->desc.max_pos, scale, ctx->status
@@ -139,6 +140,7 @@ cudaError_t launch_rows(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_
 
 cudaError_t rc_launch_decode_append(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st) {
   const int d = ctx->desc.head_dim, G = ctx->desc.n_kv_heads;
+  RcLaunchScope scope(ctx, RC_K_DECODE_APPEND, st);
   if (ctx->desc.dtype == RECACHE_BF16)
     decode_append_kernel<__nv_bfloat16><<<a.batch * G, 64, 0, st>>>(
         (const __nv_bfloat16*)a.k_new, (const __nv_bfloat16*)a.v_new, a.q_pos, (__nv_bfloat16*)a.k_pages,

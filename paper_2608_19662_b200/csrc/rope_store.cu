@@ -108,6 +108,7 @@ cudaError_t rc_launch_rope_store(const recache_ctx* ctx, const RopeStoreArgs& a,
   const int64_t n_work = (int64_t)a.total * G * chunks;
   const int threads = 256;
   const unsigned blocks = (unsigned)((n_work + threads - 1) / threads);
+  RcLaunchScope scope(ctx, RC_K_ROPE_STORE, st);
   if (bf)
     rope_store_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
         (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, (__nv_bfloat16*)a.k_dst, (__nv_bfloat16*)a.v_dst,

@@ -363,3 +363,64 @@ def keep_all(pool: ResourceBatch) -> ResourceBatch:
         keep[s:s + l] = 1
     p.keep = keep
     return p
+
+
+# --------------------------------------------------------------------------
+# Decode composed from a resource pool (paged compaction feeds the decode).
+# --------------------------------------------------------------------------
+@dataclass
+class DecodeCompose:
+    """Config-4-shaped decode where the resource pages are materialised from a
+    cache pool by paged compaction.  Only index data lives here; the cache and
+    history contents are N(0,1) tensors drawn by `seeded_normal`."""
+    shape: Shape
+    batch: int
+    lens: np.ndarray              # [batch * n_res] pool resource lengths
+    dst_slot: np.ndarray
+    pool_tokens: int
+    keep: np.ndarray              # [pool_tokens]
+    res_off: np.ndarray           # [batch + 1]
+    vis: np.ndarray               # [G][batch * n_res]
+    hist_len: np.ndarray          # [batch * G]
+    hist_page_table: np.ndarray   # [batch * G, hist_pages]
+    free_pages: np.ndarray        # page ids handed to compaction (shuffled)
+    n_pages: int
+    max_res_pages: int
+    q_pos: np.ndarray             # [batch]
+
+
+def config4_compose(batch=64, n_res=16, res_len=(500, 700), route_frac=0.25, hist=2048,
+                    seed=SEED0 + 4, shape: Shape = QWEN3_4B) -> DecodeCompose:
+    rng = np.random.default_rng(seed + 7)
+    g = shape.n_kv_heads
+    lens = uniform_lengths(rng, batch * n_res, *res_len)
+    masks = keep_mask_spans(rng, lens)
+    slot = np.zeros(len(lens), np.int32)
+    slot[1:] = np.cumsum(lens)[:-1]
+    pool_tokens = int(lens.sum())
+    keep = np.concatenate(masks).astype(np.uint8)
+    res_off = (np.arange(batch + 1) * n_res).astype(np.int32)
+    vis = np.concatenate([routes_random(rng, g, n_res, route_frac) for _ in range(batch)], axis=1)
+    kept = np.array([int(m.sum()) for m in masks])
+    route_len = np.array([[int((vis[kg, b * n_res:(b + 1) * n_res] * kept[b * n_res:(b + 1) * n_res]).sum())
+                           for kg in range(g)] for b in range(batch)]).reshape(-1)
+    res_pages = (route_len + PAGE_TOKENS - 1) // PAGE_TOKENS
+    hist_pages = (hist + PAGE_TOKENS - 1) // PAGE_TOKENS
+    n_res_pages = int(res_pages.sum())
+    n_pages = n_res_pages + batch * g * hist_pages
+    order = rng.permutation(n_pages).astype(np.int32)
+    free_pages = order[:n_res_pages].copy()
+    hpt = order[n_res_pages:].reshape(batch * g, hist_pages).copy()
+    q_pos = np.full(batch, int(lens[:n_res].sum()) + hist - 1, np.int32)
+    return DecodeCompose(shape, batch, lens, slot, pool_tokens, keep, res_off, np.ascontiguousarray(vis),
+                         np.full(batch * g, hist, np.int32), hpt, free_pages, n_pages,
+                         int(res_pages.max()) if len(res_pages) else 1, q_pos)
+
+
+def seeded_normal(seed: int, shape, dtype: torch.dtype, device="cpu") -> torch.Tensor:
+    """N(0,1) from a seeded generator on `device` (cache / page contents that
+    stand in for earlier encode results; drawn where they are used)."""
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) & 0x7FFFFFFFFFFFFFFF)
+    return torch.randn(*shape, generator=g, dtype=torch.float32 if device == "cpu" else dtype,
+                       device=device).to(dtype)
