@@ -87,6 +87,7 @@ class Workload:
         n_res = len(dc.lens) // dc.batch
         rl4 = np.array([[int((dc.vis[kg, b * n_res:(b + 1) * n_res] * kept4[b * n_res:(b + 1) * n_res]).sum())
                          for kg in range(g)] for b in range(dc.batch)]).reshape(-1)
+        self.dec_res_rows = int(rl4.sum())
         self.dec_rows = int(rl4.sum() + dc.hist_len.sum())
         self.pairs_decode = self.dec_rows * sh.group_size
         self.flops = {k: 4 * d * v for k, v in (("encode", self.pairs_encode), ("prefill", self.pairs_prefill),
@@ -145,7 +146,7 @@ class Runner:
         n_items = dc.batch * g
         self.d_route_cu = E(n_items + 1, dtype=torch.int32)
         self.d_route_len = E(n_items, dtype=torch.int32)
-        self.d_route_idx = E(int(dc.keep.sum()) * 1 + 64, dtype=torch.int32)
+        self.d_route_idx = E(w.dec_res_rows + 64, dtype=torch.int32)
         self.d_page_table = E(n_items, dc.max_res_pages, dtype=torch.int32)
         self.o_dec = E(dc.batch, sh.n_q_heads, d)
         rc = self.rc

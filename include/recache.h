@@ -76,7 +76,8 @@ enum {
   RECACHE_DEV_OVERFLOW = 3,     /* route rows exceed row_capacity */
   RECACHE_DEV_BAD_PAGE = 4,     /* page id outside [0, n_pages) or table too short */
   RECACHE_DEV_NO_PAGES = 5,     /* free page list exhausted */
-  RECACHE_DEV_BAD_POS = 6       /* position outside [0, max_pos) */
+  RECACHE_DEV_BAD_POS = 6,      /* position outside [0, max_pos) */
+  RECACHE_DEV_TIMEOUT = 7       /* a kernel gave up waiting on one of its own barriers */
 };
 
 typedef struct recache_ctx recache_ctx;

@@ -148,3 +148,17 @@ int64_t rc_decode_workspace_bytes(const recache_ctx* ctx, int batch, int max_res
 cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, cudaStream_t st);
 cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a, cudaStream_t st);
 cudaError_t rc_launch_decode(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
+
+// ---- bf16 tensor-core attention (tcgen05 / TMEM / TMA) ----
+struct TcAttnArgs {
+  const void* q; void* o; int out_dtype;
+  const int32_t* cu; int n_seq; int total; int max_len;
+  const int32_t* pos0;                     // null: positions start at 0
+  const int32_t* slot;                     // null: causal rows start at cu[b]
+  const void* k_self; const void* v_self; int64_t self_rows;   // [G][self_rows][128]
+  const void* k_route; const void* v_route; const int32_t* route_cu; int64_t route_rows;
+  void* workspace;
+};
+bool rc_tc_supported(const recache_ctx* ctx);
+int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);
+cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaStream_t st);

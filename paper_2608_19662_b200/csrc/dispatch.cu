@@ -1,17 +1,34 @@
 // Chooses the kernel for each attention call and sizes its scratch.
+//   fp32 contexts, and bf16 shapes the tensor-core kernel does not cover
+//   (head_dim 64, one or more than eight query heads per group): exact row kernels.
+//   bf16, head_dim 128, 2/4/8 query heads per group: tcgen05 kernel.
 #include "common.cuh"
 
-int64_t rc_encode_workspace_bytes(const recache_ctx*, int, int, int) { return 0; }
-int64_t rc_prefill_workspace_bytes(const recache_ctx*, int, int, int) { return 0; }
+int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, int max_len) {
+  return rc_tc_supported(ctx) ? rc_tc_workspace_bytes(ctx, n_res, total, max_len) : 0;
+}
+int64_t rc_prefill_workspace_bytes(const recache_ctx* ctx, int n_req, int total_q, int max_q) {
+  return rc_tc_supported(ctx) ? rc_tc_workspace_bytes(ctx, n_req, total_q, max_q) : 0;
+}
 int64_t rc_decode_workspace_bytes(const recache_ctx*, int, int, int) { return 0; }
 
 cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, cudaStream_t st) {
+  if (rc_tc_supported(ctx)) {
+    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, a.max_len, nullptr, a.slot, a.k_cache, a.v_cache,
+                 a.pool_tokens, nullptr, nullptr, nullptr, 0, a.workspace};
+    return rc_launch_attn_tc(ctx, t, st);
+  }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, nullptr, a.slot, a.k_cache, a.v_cache,
                  a.pool_tokens, nullptr, nullptr, nullptr};
   return rc_launch_attn_rows(ctx, r, st);
 }
 
 cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a, cudaStream_t st) {
+  if (rc_tc_supported(ctx)) {
+    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.max_q, a.pos0, nullptr, a.k_conv, a.v_conv,
+                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace};
+    return rc_launch_attn_tc(ctx, t, st);
+  }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, nullptr, a.k_conv, a.v_conv,
                  (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu};
   return rc_launch_attn_rows(ctx, r, st);
