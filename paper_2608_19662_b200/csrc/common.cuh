@@ -162,3 +162,8 @@ struct TcAttnArgs {
 bool rc_tc_supported(const recache_ctx* ctx);
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);
 cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaStream_t st);
+
+// ---- bf16 split-KV paged decode (TMA + mma.sync, persistent) ----
+bool rc_decode_split_supported(const recache_ctx* ctx);
+int64_t rc_decode_split_workspace_bytes(const recache_ctx* ctx, int batch, int max_res_pages, int max_hist_pages);
+cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);

@@ -1,0 +1,474 @@
+// Routed split-KV decode for bf16, head_dim 128, 64-token pages: memory-bound.
+//
+// Persistent kernel, one CTA per SM.  A work unit is (item = sequence x KV group,
+// split) = a contiguous range of the item's logical pages (resource pages first,
+// then history pages).  Units are dealt round-robin to the CTAs.  Inside a CTA
+//   warp 3     : TMA producer.  Walks its units' pages in order and keeps a ring
+//                of NSTAGE (K page + V page) buffers full; it runs ahead across
+//                unit boundaries, so the HBM stream never drains.
+//   warps 0-2  : consumers.  The page at ring position n belongs to warp n % 3
+//                and stage n % 6, so a stage is always consumed by the same warp
+//                and that warp sees every phase of its stages' barriers in
+//                order (a parity wait is only valid one phase ahead).  The s
+//                query heads of the group are the first s rows of a 16-row
+//                mma.sync tile, so each K/V byte is read once for all heads.
+//                Scores: m16n8k16 over ldmatrix fragments of the swizzled K page;
+//                online softmax in registers (quad shuffles); O += P V with
+//                transposed ldmatrix fragments of the V page.
+// The consumer warps' partial (max, sum, O) are merged through shared memory; with
+// more than one split the unit's partial goes to the workspace and a second
+// small kernel merges the splits.
+// Every K/V byte crosses HBM once; the roofline is bytes / HBM bandwidth.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int D = 128;
+constexpr int PT = 64;                 // tokens per page
+constexpr int NSTAGE = 6;
+constexpr int PAGE_BYTES = PT * D * 2; // 16 KB
+constexpr int BOX_BYTES = 8192;        // [64 tokens][64 bf16], 128-byte swizzle
+constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+constexpr int NCW = 3;                 // consumer warps; NSTAGE % NCW == 0
+static_assert(NSTAGE % NCW == 0, "a stage must always be consumed by the same warp");
+constexpr int NTHREADS = (NCW + 1) * 32;
+constexpr int SM_STAGES = 0;
+constexpr int SM_BAR = NSTAGE * STAGE_BYTES;          // full[NSTAGE], empty[NSTAGE]
+constexpr int SM_Q = SM_BAR + 2 * NSTAGE * 8 + 32;    // per-warp rotated q: NCW x 8 x 128 bf16
+constexpr int SM_MERGE = SM_Q + NCW * 8 * D * 2;      // NCW x 8 x (2 + 128) floats
+constexpr int SM_MISC = SM_MERGE + NCW * 8 * 130 * 4;
+constexpr int SM_TOTAL = SM_MISC + 64;
+constexpr int SM_ALLOC = SM_TOTAL + 1024;
+constexpr long long WAIT_CYCLES = 4000000000ll;
+
+struct DecParams {
+  const __nv_bfloat16* q; const int32_t* q_pos;
+  const int32_t* res_pt; int max_res_pages; const int32_t* res_len;
+  const int32_t* hist_pt; int max_hist_pages; const int32_t* hist_len;
+  int n_items, n_splits, G, Hq, s;
+  int64_t n_pages;
+  void* out; float* part_o; float* part_ml;      // partials: [unit][s][128], [unit][s][2]
+  const float* cos_tab; const float* sin_tab; int max_pos;
+  float scale_log2;
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait (see the tensor-core attention kernel): never spins forever.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try(bar, parity)) return;
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return;
+    if ((it & 63) == 63) {
+      if (*abort_flag) return;
+      if (clock64() - t0 > WAIT_CYCLES) { *abort_flag = 1; rc_set_status(status, RECACHE_DEV_TIMEOUT); return; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
+
+// Pages of item `it` and the range split `sp` owns.
+struct UnitPages { int n_res_pages, n_hist_pages, p0, p1, res_len, hist_len; };
+__device__ __forceinline__ UnitPages unit_pages(const DecParams& p, int it, int sp) {
+  UnitPages u;
+  u.res_len = max(p.res_len[it], 0);
+  u.hist_len = max(p.hist_len[it], 0);
+  u.n_res_pages = min((u.res_len + PT - 1) / PT, p.max_res_pages);
+  u.n_hist_pages = min((u.hist_len + PT - 1) / PT, p.max_hist_pages);
+  const int total = u.n_res_pages + u.n_hist_pages;
+  u.p0 = (int)((int64_t)total * sp / p.n_splits);
+  u.p1 = (int)((int64_t)total * (sp + 1) / p.n_splits);
+  return u;
+}
+
+template <typename TO>
+__global__ void __launch_bounds__(NTHREADS, 1) decode_split_kernel(const __grid_constant__ CUtensorMap tm_k,
+                                                                   const __grid_constant__ CUtensorMap tm_v,
+                                                                   const DecParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t sm = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sm_gen = smem_raw + (sm - smem_u32(smem_raw));
+  const uint32_t bars = sm + SM_BAR;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_gen + SM_MISC);
+  auto full = [&](int i) { return bars + 8u * (uint32_t)i; };
+  auto empty = [&](int i) { return bars + 8u * (uint32_t)(NSTAGE + i); };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_units = p.n_items * p.n_splits;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < NSTAGE; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == NCW) {
+    // ===================== producer =====================
+    if (lane == 0) {
+      uint32_t n = 0;   // pages issued so far (ring position)
+      for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        const int it = unit / p.n_splits, sp = unit % p.n_splits;
+        const UnitPages u = unit_pages(p, it, sp);
+        for (int lp = u.p0; lp < u.p1; ++lp, ++n) {
+          int pg = lp < u.n_res_pages ? p.res_pt[(int64_t)it * p.max_res_pages + lp]
+                                      : p.hist_pt[(int64_t)it * p.max_hist_pages + (lp - u.n_res_pages)];
+          if (pg < 0 || pg >= p.n_pages) { rc_set_status(p.status, RECACHE_DEV_BAD_PAGE); pg = 0; }
+          const int st = n % NSTAGE;
+          mbar_wait(empty(st), ((n / NSTAGE) & 1u) ^ 1u, abort_flag, p.status);
+          mbar_expect_tx(full(st), STAGE_BYTES);
+          const uint32_t dst = sm + SM_STAGES + st * STAGE_BYTES;
+          tma_load_2d(dst, &tm_k, full(st), 0, pg * PT);
+          tma_load_2d(dst + BOX_BYTES, &tm_k, full(st), 64, pg * PT);
+          tma_load_2d(dst + PAGE_BYTES, &tm_v, full(st), 0, pg * PT);
+          tma_load_2d(dst + PAGE_BYTES + BOX_BYTES, &tm_v, full(st), 64, pg * PT);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ===================== consumers =====================
+    const int gq = lane >> 2, tq = lane & 3;           // fragment row (query head) and column pair
+    const int s = p.s;
+    uint32_t n_base = 0;                                // ring position of the unit's first page
+    __nv_bfloat16* q_sm = reinterpret_cast<__nv_bfloat16*>(sm_gen + SM_Q) + warp * 8 * D;
+    float* mrg = reinterpret_cast<float*>(sm_gen + SM_MERGE);
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+      const int it = unit / p.n_splits, sp = unit % p.n_splits;
+      const int b = it / p.G, g = it % p.G;
+      const UnitPages u = unit_pages(p, it, sp);
+      if (sp == 0 && lane == 0 && warp == 0) {
+        if (u.hist_len < 1 || (u.res_len + PT - 1) / PT > p.max_res_pages || (u.hist_len + PT - 1) / PT > p.max_hist_pages)
+          rc_set_status(p.status, RECACHE_DEV_BAD_PAGE);
+      }
+      // ---- rotated query heads of the group -> A fragments (rows >= s are zero) ----
+      {
+        int pos = p.q_pos[b];
+        if (pos < 0 || pos >= p.max_pos) { rc_set_status(p.status, RECACHE_DEV_BAD_POS); pos = min(max(pos, 0), p.max_pos - 1); }
+        const __nv_bfloat16* qg = p.q + ((int64_t)b * p.Hq + g * s) * D;
+        for (int e = lane; e < 8 * 64; e += 32) {
+          const int h = e >> 6, i = e & 63;
+          float olo = 0.f, ohi = 0.f;
+          if (h < s) {
+            const float lo = __bfloat162float(qg[h * D + i]), hi = __bfloat162float(qg[h * D + i + 64]);
+            const float c = p.cos_tab[(int64_t)pos * 64 + i], sn = p.sin_tab[(int64_t)pos * 64 + i];
+            olo = __fmaf_rn(lo, c, -__fmul_rn(hi, sn));
+            ohi = __fmaf_rn(hi, c, __fmul_rn(lo, sn));
+          }
+          q_sm[h * D + i] = __float2bfloat16_rn(olo);
+          q_sm[h * D + i + 64] = __float2bfloat16_rn(ohi);
+        }
+        __syncwarp();
+      }
+      uint32_t qa[8][2];   // per k-step: a0 (cols 2tq,+1) and a2 (cols 8+2tq,+1) of row gq; rows 8..15 are zero
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        qa[kk][0] = *reinterpret_cast<const uint32_t*>(q_sm + gq * D + kk * 16 + tq * 2);
+        qa[kk][1] = *reinterpret_cast<const uint32_t*>(q_sm + gq * D + kk * 16 + 8 + tq * 2);
+      }
+      __syncwarp();
+
+      float o[16][4];
+#pragma unroll
+      for (int nt = 0; nt < 16; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+      float m_run = -INFINITY, l_run = 0.f;      // row gq (replicated over the quad), log2 domain
+
+      // first page of the unit whose ring position belongs to this warp
+      const int first = (int)(((uint32_t)warp + NCW - n_base % NCW) % NCW);
+      for (int lp = u.p0 + first; lp < u.p1; lp += NCW) {
+        const uint32_t n = n_base + (uint32_t)(lp - u.p0);
+        const int st = n % NSTAGE;
+        // tokens of this page that exist
+        int valid = PT;
+        if (lp < u.n_res_pages) valid = min(PT, u.res_len - lp * PT);
+        else valid = min(PT, u.hist_len - (lp - u.n_res_pages) * PT);
+        mbar_wait(full(st), (n / NSTAGE) & 1u, abort_flag, p.status);
+        const uint32_t kb = sm + SM_STAGES + st * STAGE_BYTES, vb = kb + PAGE_BYTES;
+        if (valid < PT) {
+          // slots past the end of the part were never written: clear their values (0 * NaN would poison O)
+          uint8_t* vg = sm_gen + SM_STAGES + st * STAGE_BYTES + PAGE_BYTES;
+          const int v0 = max(valid, 0);
+          for (int e = lane; e < (PT - v0) * 16; e += 32) {
+            const int r = v0 + (e >> 4), c = e & 15;
+            *reinterpret_cast<uint4*>(vg + (c >> 3) * BOX_BYTES + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // a later TMA load overwrites these bytes
+          __syncwarp();
+        }
+        // ---- S = q K^T : 8 token tiles x 8 k-steps ----
+        float sc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+          const int tok = nt * 8 + (lane & 7);
+#pragma unroll
+          for (int kq = 0; kq < 4; ++kq) {
+            const int c = 4 * kq + (lane >> 3);
+            const uint32_t addr = kb + (c >> 3) * BOX_BYTES + tok * 128 + (((c & 7) ^ (tok & 7)) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(addr, b0, b1, b2, b3);
+            mma_bf16(sc[nt], qa[2 * kq][0], 0u, qa[2 * kq][1], 0u, b0, b1);
+            mma_bf16(sc[nt], qa[2 * kq + 1][0], 0u, qa[2 * kq + 1][1], 0u, b2, b3);
+          }
+        }
+        // ---- online softmax of row gq (columns nt*8 + 2tq, +1) ----
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          const int c0 = nt * 8 + tq * 2;
+          sc[nt][0] = c0 < valid ? sc[nt][0] * p.scale_log2 : -INFINITY;
+          sc[nt][1] = c0 + 1 < valid ? sc[nt][1] * p.scale_log2 : -INFINITY;
+          mx = fmaxf(mx, fmaxf(sc[nt][0], sc[nt][1]));
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        const float m_use = m_new == -INFINITY ? 0.f : m_new;    // a page with no valid token
+        const float corr = ex2(m_run - m_use);                   // 0 on the first page
+        float ps = 0.f;
+        uint32_t pa[4][2];   // P as A fragments: per 16-token k-step, a0 / a2 of row gq
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          const float p0 = ex2(sc[nt][0] - m_use), p1 = ex2(sc[nt][1] - m_use);
+          ps += p0 + p1;
+          pa[nt >> 1][nt & 1] = pack2(p0, p1);
+        }
+        ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+        ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+        l_run = l_run * corr + ps;
+        m_run = m_new;
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= corr; o[nt][1] *= corr; }
+        // ---- O += P V : 4 k-steps (16 tokens) x 16 d tiles ----
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const int tok = kk * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+          for (int np = 0; np < 8; ++np) {
+            const int c = 2 * np + (lane >> 4);
+            const uint32_t addr = vb + (c >> 3) * BOX_BYTES + tok * 128 + (((c & 7) ^ (tok & 7)) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4_t(addr, b0, b1, b2, b3);
+            mma_bf16(o[2 * np], pa[kk][0], 0u, pa[kk][1], 0u, b0, b1);
+            mma_bf16(o[2 * np + 1], pa[kk][0], 0u, pa[kk][1], 0u, b2, b3);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty(st));
+      }
+      n_base += (uint32_t)(u.p1 - u.p0);
+
+      // ---- merge the consumer warps' partials (rows gq < s) ----
+      if (gq < s) {
+        float* mine = mrg + (warp * 8 + gq) * 130;
+        if (tq == 0) { mine[0] = m_run; mine[1] = l_run; }
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+          mine[2 + nt * 8 + tq * 2] = o[nt][0];
+          mine[2 + nt * 8 + tq * 2 + 1] = o[nt][1];
+        }
+      }
+      bar_consumers();
+      {
+        const int t = threadIdx.x;               // head t/32 (+NCW ...), dims (t%32)*4..+3
+        for (int h = t >> 5; h < s; h += NCW) {
+          float mw[NCW], M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) { mw[w] = mrg[(w * 8 + h) * 130]; M = fmaxf(M, mw[w]); }
+          float Lsum = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int w = 0; w < NCW; ++w) {
+            const float f = mw[w] == -INFINITY ? 0.f : ex2(mw[w] - M);
+            Lsum += mrg[(w * 8 + h) * 130 + 1] * f;
+            const float* ow = mrg + (w * 8 + h) * 130 + 2 + (t & 31) * 4;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[c] += ow[c] * f;
+          }
+          if (p.n_splits == 1) {
+            const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+            TO* orow = reinterpret_cast<TO*>(p.out) + ((int64_t)b * p.Hq + g * s + h) * D + (t & 31) * 4;
+            if constexpr (sizeof(TO) == 4) {
+              *reinterpret_cast<float4*>(orow) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+            } else {
+              *reinterpret_cast<uint2*>(orow) = make_uint2(pack2(acc[0] * inv, acc[1] * inv), pack2(acc[2] * inv, acc[3] * inv));
+            }
+          } else {
+            float* po = p.part_o + ((int64_t)unit * s + h) * D + (t & 31) * 4;
+            *reinterpret_cast<float4*>(po) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            if ((t & 31) == 0) { p.part_ml[((int64_t)unit * s + h) * 2] = M; p.part_ml[((int64_t)unit * s + h) * 2 + 1] = Lsum; }
+          }
+        }
+      }
+      bar_consumers();
+    }
+  }
+}
+
+// Combines the splits of every (sequence, head): grid = batch * Hq, 32 threads x 4 dims.
+template <typename TO>
+__global__ void __launch_bounds__(32) decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                                          TO* __restrict__ out, int n_splits, int G, int Hq, int s) {
+  const int row = blockIdx.x;                 // b * Hq + head
+  const int b = row / Hq, head = row % Hq, g = head / s, h = head % s;
+  const int it = b * G + g;
+  const int t = threadIdx.x;
+  float M = -INFINITY;
+  for (int sp = 0; sp < n_splits; ++sp) M = fmaxf(M, part_ml[((int64_t)(it * n_splits + sp) * s + h) * 2]);
+  float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int sp = 0; sp < n_splits; ++sp) {
+    const int64_t u = ((int64_t)(it * n_splits + sp) * s + h);
+    const float mw = part_ml[u * 2];
+    const float f = mw == -INFINITY ? 0.f : ex2(mw - M);
+    L += part_ml[u * 2 + 1] * f;
+    const float4 v = *reinterpret_cast<const float4*>(part_o + u * D + t * 4);
+    acc[0] += v.x * f; acc[1] += v.y * f; acc[2] += v.z * f; acc[3] += v.w * f;
+  }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  TO* orow = out + (int64_t)row * D + t * 4;
+  if constexpr (sizeof(TO) == 4) {
+    *reinterpret_cast<float4*>(orow) = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+  } else {
+    *reinterpret_cast<uint2*>(orow) = make_uint2(pack2(acc[0] * inv, acc[1] * inv), pack2(acc[2] * inv, acc[3] * inv));
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  }
+  return fn;
+}
+// page pool viewed as [n_pages * 64 rows][128 bf16]; box = one page x 64 columns
+bool map_pages(CUtensorMap* m, const void* base, uint64_t n_pages) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {128, n_pages * PT};
+  cuuint64_t strides[1] = {256};
+  cuuint32_t box[2] = {64, PT};
+  cuuint32_t es[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
+
+}  // namespace
+
+bool rc_decode_split_supported(const recache_ctx* ctx) {
+  const int s = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;
+  return ctx->desc.dtype == RECACHE_BF16 && ctx->desc.head_dim == 128 && ctx->desc.page_tokens == PT && s <= 8;
+}
+
+// Splits per item: the smallest count that fills the persistent grid evenly
+// (units / SMs close to an integer from below) while a split keeps >= 4 pages.
+int rc_decode_n_splits(const recache_ctx* ctx, int batch, int max_res_pages, int max_hist_pages) {
+  const int items = batch * ctx->desc.n_kv_heads, sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+  const int pages = max_res_pages + max_hist_pages;
+  int best = 1; double best_eff = 0.0;
+  for (int ns = 1; ns <= 16; ++ns) {
+    if (ns > 1 && pages / ns < 4) break;
+    const int units = items * ns;
+    const double eff = (double)units / ((double)((units + sms - 1) / sms) * sms);
+    if (eff > best_eff + 0.02) { best_eff = eff; best = ns; }
+  }
+  return best;
+}
+
+int64_t rc_decode_split_workspace_bytes(const recache_ctx* ctx, int batch, int max_res_pages, int max_hist_pages) {
+  const int ns = rc_decode_n_splits(ctx, batch, max_res_pages, max_hist_pages);
+  const int s = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;
+  const int64_t units = (int64_t)batch * ctx->desc.n_kv_heads * ns;
+  return align256(units * s * D * 4) + align256(units * s * 2 * 4);
+}
+
+cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st) {
+  const int G = ctx->desc.n_kv_heads, Hq = ctx->desc.n_q_heads, s = Hq / G;
+  const int ns = rc_decode_n_splits(ctx, a.batch, a.max_res_pages, a.max_hist_pages);
+  const int64_t units = (int64_t)a.batch * G * ns;
+  CUtensorMap tk, tv;
+  if (!map_pages(&tk, a.k_pages, (uint64_t)a.n_pages) || !map_pages(&tv, a.v_pages, (uint64_t)a.n_pages))
+    return cudaErrorInvalidValue;
+  DecParams p;
+  p.q = (const __nv_bfloat16*)a.q; p.q_pos = a.q_pos;
+  p.res_pt = a.res_pt; p.max_res_pages = a.max_res_pages; p.res_len = a.res_len;
+  p.hist_pt = a.hist_pt; p.max_hist_pages = a.max_hist_pages; p.hist_len = a.hist_len;
+  p.n_items = a.batch * G; p.n_splits = ns; p.G = G; p.Hq = Hq; p.s = s; p.n_pages = a.n_pages;
+  p.out = a.o;
+  p.part_o = (float*)a.workspace;
+  p.part_ml = (float*)((uint8_t*)a.workspace + align256(units * s * D * 4));
+  p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
+  p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
+  p.status = ctx->status;
+  const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+  const unsigned grid = (unsigned)(units < sms ? units : sms);
+  const bool f32 = a.out_dtype == RECACHE_F32;
+  {
+    RcLaunchScope scope(ctx, RC_K_DECODE_ATTN, st);
+    if (f32) {
+      static bool done = false;
+      if (!done) { cudaFuncSetAttribute(decode_split_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); done = true; }
+      decode_split_kernel<float><<<grid, NTHREADS, SM_ALLOC, st>>>(tk, tv, p);
+    } else {
+      static bool done = false;
+      if (!done) { cudaFuncSetAttribute(decode_split_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); done = true; }
+      decode_split_kernel<__nv_bfloat16><<<grid, NTHREADS, SM_ALLOC, st>>>(tk, tv, p);
+    }
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || ns == 1) return e;
+  RcLaunchScope scope(ctx, RC_K_DECODE_MERGE, st);
+  if (f32) decode_merge_kernel<float><<<a.batch * Hq, 32, 0, st>>>(p.part_o, p.part_ml, (float*)a.o, ns, G, Hq, s);
+  else decode_merge_kernel<__nv_bfloat16><<<a.batch * Hq, 32, 0, st>>>(p.part_o, p.part_ml, (__nv_bfloat16*)a.o, ns, G, Hq, s);
+  return cudaGetLastError();
+}

@@ -2,6 +2,7 @@
 //   fp32 contexts, and bf16 shapes the tensor-core kernel does not cover
 //   (head_dim 64, one or more than eight query heads per group): exact row kernels.
 //   bf16, head_dim 128, 2/4/8 query heads per group: tcgen05 kernel.
+//   bf16 decode, head_dim 128, 64-token pages, <= 8 heads per group: split-KV kernel.
 #include "common.cuh"
 
 int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, int max_len) {
@@ -10,7 +11,9 @@ int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, 
 int64_t rc_prefill_workspace_bytes(const recache_ctx* ctx, int n_req, int total_q, int max_q) {
   return rc_tc_supported(ctx) ? rc_tc_workspace_bytes(ctx, n_req, total_q, max_q) : 0;
 }
-int64_t rc_decode_workspace_bytes(const recache_ctx*, int, int, int) { return 0; }
+int64_t rc_decode_workspace_bytes(const recache_ctx* ctx, int batch, int max_res_pages, int max_hist_pages) {
+  return rc_decode_split_supported(ctx) ? rc_decode_split_workspace_bytes(ctx, batch, max_res_pages, max_hist_pages) : 0;
+}
 
 cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, cudaStream_t st) {
   if (rc_tc_supported(ctx)) {
@@ -35,5 +38,6 @@ cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a,
 }
 
 cudaError_t rc_launch_decode(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st) {
+  if (rc_decode_split_supported(ctx)) return rc_launch_decode_split(ctx, a, st);
   return rc_launch_decode_rows(ctx, a, st);
 }
