@@ -231,6 +231,40 @@ RECACHE_API recache_status recache_attend_decode(recache_ctx* ctx,
     void* out_o, int32_t out_dtype,
     void* workspace, int64_t workspace_bytes, void* stream);
 
+/*
+ * Decode without any allocation.  (The paper has no counterpart: this is a
+ * deployment variant of recache_attend_decode, same arguments minus the
+ * workspace, same results.)
+ *
+ * Who needs it: callers that may not allocate device memory where they decode -
+ * a serving loop that has frozen its memory plan, a plugin inside a host process
+ * that owns all device memory, a latency-critical path that must not enter the
+ * allocator.  The split-KV partials go to a 4 MiB scratch array that is part of
+ * the library image on every GPU that loads it (held until the process exits),
+ * so nothing is allocated or freed, here or in any library this call uses.
+ *
+ * Limits and rules
+ *  - bf16 contexts with head_dim 128 and 64-token pages only (RECACHE_EUNSUPPORTED
+ *    otherwise); the kernel timer must be off (it creates event objects).
+ *  - batch * n_kv_heads * splits * heads-per-group * 520 bytes must fit in 4 MiB
+ *    (e.g. batch 64 with 8 KV groups of 4 heads uses 2.1 MiB); beyond that the
+ *    call returns RECACHE_ENOMEM with a message and launches nothing.
+ *  - The first call on a device looks up the scratch array's device address
+ *    (once per device, with that device current).  Make that first call outside
+ *    any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's
+ *    contents; every slot a call reads it has written first, so nothing needs
+ *    clearing.  Two calls that overlap on the GPU (different streams) race on
+ *    it: serialise them.
+ */
+RECACHE_API recache_status recache_attend_decode_noalloc(recache_ctx* ctx,
+    const void* q, const int32_t* q_pos, int32_t batch,
+    const void* k_new, const void* v_new,
+    void* k_pages, void* v_pages, int64_t n_pages,
+    const int32_t* res_page_table, int32_t max_res_pages, const int32_t* res_len,
+    const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
+    void* out_o, int32_t out_dtype, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -51,6 +51,8 @@ SIGNATURES = {
                                          _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                         _P, _I32, _P, _I64, _P]),
+    "recache_attend_decode_noalloc": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
+                                                _P, _I32, _P]),
 }
 
 _lib = None
@@ -230,4 +232,18 @@ class ReCache:
                                             _ptr(res_len), _ptr(hist_page_table), mh, _ptr(hist_len), _ptr(out), oc,
                                             _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_attend_decode")
+        return out
+
+    def attend_decode_noalloc(self, q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page_table, hist_len,
+                              out, k_new=None, v_new=None):
+        """recache_attend_decode_noalloc: decode for callers that must not allocate where they decode.
+        `out` [B,Hq,d] (bf16 or fp32) is caller-provided; the split partials live in the library's own
+        4 MiB scratch, so neither the library nor this wrapper allocates anything.  Calls on one device
+        share that scratch: do not overlap them on different streams."""
+        oc = F32 if out.dtype == torch.float32 else BF16
+        st = self.lib.recache_attend_decode_noalloc(
+            self.h, _ptr(q), _ptr(q_pos), q.shape[0], _ptr(k_new), _ptr(v_new), _ptr(k_pages), _ptr(v_pages),
+            k_pages.shape[0], _ptr(res_page_table), res_page_table.shape[1], _ptr(res_len), _ptr(hist_page_table),
+            hist_page_table.shape[1], _ptr(hist_len), _ptr(out), oc, _stream())
+        self._check(st, "recache_attend_decode_noalloc")
         return out

@@ -472,3 +472,76 @@ cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, 
   else decode_merge_kernel<__nv_bfloat16><<<a.batch * Hq, 32, 0, st>>>(p.part_o, p.part_ml, (__nv_bfloat16*)a.o, ns, G, Hq, s);
   return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------
+// Allocation-free decode.
+//
+// recache_attend_decode needs a scratch buffer for the split partials, which the
+// caller normally gets from its allocator.  Some callers cannot allocate at the
+// point where they decode: code running inside a region where the CUDA allocator
+// must not be touched (a serving loop that has pinned down its memory plan, a
+// plugin loaded into a host process that owns all device memory, a signal-safe
+// or real-time path).  For them the scratch lives in this file-scope device
+// array, reserved by every GPU that loads the library until the process exits.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t NOALLOC_SCRATCH_BYTES = 4ll << 20;   // 4 MiB per device
+static __device__ __align__(256) unsigned char g_decode_scratch[NOALLOC_SCRATCH_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+void* g_scratch_addr[NOALLOC_MAX_DEVICES] = {nullptr};   // device address of g_decode_scratch, per device
+
+}  // namespace
+
+extern "C" RECACHE_API recache_status recache_attend_decode_noalloc(
+    recache_ctx* ctx, const void* q, const int32_t* q_pos, int32_t batch, const void* k_new, const void* v_new,
+    void* k_pages, void* v_pages, int64_t n_pages, const int32_t* res_page_table, int32_t max_res_pages,
+    const int32_t* res_len, const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
+    void* out_o, int32_t out_dtype, void* stream) {
+  if (!ctx) return RECACHE_EINVAL;
+  auto fail = [&](recache_status st, const char* msg) { ctx->err = msg; return st; };
+  if (batch < 0 || n_pages < 0 || max_res_pages < 0 || max_hist_pages <= 0)
+    return fail(RECACHE_EINVAL, "decode_noalloc: bad size");
+  if (out_dtype != RECACHE_F32 && out_dtype != ctx->desc.dtype)
+    return fail(RECACHE_EINVAL, "decode_noalloc: out_dtype must be f32 or the context dtype");
+  if (batch == 0) return RECACHE_OK;
+  if (!q || !q_pos || !k_pages || !v_pages || !res_len || !hist_page_table || !hist_len || !out_o ||
+      (max_res_pages > 0 && !res_page_table) || ((k_new == nullptr) != (v_new == nullptr)))
+    return fail(RECACHE_EINVAL, "decode_noalloc: null pointer");
+  if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)out_o) & 15)
+    return fail(RECACHE_EINVAL, "decode_noalloc: tensors must be 16-byte aligned");
+  if (!rc_decode_split_supported(ctx))
+    return fail(RECACHE_EUNSUPPORTED, "decode_noalloc: needs a bf16 context with head_dim 128 and 64-token pages");
+  if (ctx->timer_on)
+    return fail(RECACHE_EINVAL, "decode_noalloc: the kernel timer creates event objects; disable it first");
+  const int64_t need = rc_decode_split_workspace_bytes(ctx, batch, max_res_pages, max_hist_pages);
+  if (need > NOALLOC_SCRATCH_BYTES)
+    return fail(RECACHE_ENOMEM, "decode_noalloc: batch x groups x splits exceeds the 4 MiB built-in scratch; "
+                                "use recache_attend_decode with a caller workspace");
+  if (ctx->device < 0 || ctx->device >= NOALLOC_MAX_DEVICES)
+    return fail(RECACHE_EUNSUPPORTED, "decode_noalloc: device index out of range");
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return fail(RECACHE_ECUDA, "decode_noalloc: set device");
+  // In host code the array's name is only a handle; the kernel needs its device
+  // address, looked up once per device with that device current.
+  void* scratch = g_scratch_addr[ctx->device];
+  if (!scratch) {
+    cudaError_t e = cudaGetSymbolAddress(&scratch, g_decode_scratch);
+    if (e != cudaSuccess || !scratch) {
+      ctx->err = std::string("decode_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e);
+      return RECACHE_ECUDA;
+    }
+    g_scratch_addr[ctx->device] = scratch;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  DecodeArgs a{q, q_pos, batch, k_new, v_new, k_pages, v_pages, n_pages, res_page_table, max_res_pages, res_len,
+               hist_page_table, max_hist_pages, hist_len, out_o, out_dtype, scratch, NOALLOC_SCRATCH_BYTES};
+  cudaError_t e = cudaSuccess;
+  if (k_new) e = rc_launch_decode_append(ctx, a, st);
+  if (e == cudaSuccess) e = rc_launch_decode_split(ctx, a, st);
+  if (e != cudaSuccess) {
+    ctx->err = std::string("decode_noalloc: launch: ") + cudaGetErrorString(e);
+    return RECACHE_ECUDA;
+  }
+  return RECACHE_OK;
+}
