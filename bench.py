@@ -18,7 +18,7 @@ e2e     = the same with every step's inputs copied from pinned host memory and
 roofline= dominant kernel (the encode attention) against the measured bf16 peak;
           `stages` also reports decode and compaction against measured HBM bandwidth.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--small]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--case full|medium|small]
 Under torchrun every rank runs an independent replica (the path has no exchange
 step); the value is the sum over ranks divided by the slowest rank's time.
 """
@@ -57,10 +57,15 @@ def load_peaks():
 class Workload:
     """Host-side (pinned) inputs + the algorithmic work they amount to."""
 
-    def __init__(self, small: bool, seed_shift: int = 0):
+    def __init__(self, case: str, seed_shift: int = 0):
         sh = wl.QWEN3_4B
         self.shape = sh
-        if small:
+        small = case == "small"
+        if case == "medium":   # profiler captures: inputs larger than L2, well under a GB on the device
+            self.pool, self.req = wl.config5(n_res=16, tq=1024, seed=wl.SEED0 + 5 + seed_shift)
+            self.dc = wl.config4_compose(batch=16, seed=wl.SEED0 + 4 + seed_shift)
+            self.name = "medium: 16 resources U[1000,2000] + 1024-token prefill; decode batch 16"
+        elif small:
             self.pool, self.req = wl.config5(n_res=6, len_range=(300, 700), tq=256, seed=wl.SEED0 + 5 + seed_shift)
             self.dc = wl.config4_compose(batch=4, n_res=8, res_len=(100, 260), hist=300, seed=wl.SEED0 + 4 + seed_shift)
             self.name = "small: 6 resources U[300,700] + 256-token prefill; decode batch 4"
@@ -283,7 +288,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = Workload(args.small)
+    w = Workload(args.case)
     for _ in range(args.warmup):
         oracle_sample(w)
     t0 = time.perf_counter(); fl = 0
@@ -310,7 +315,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--small", action="store_true", help="a small case (for profiler captures)")
+    ap.add_argument("--case", default="full", choices=["full", "medium", "small"],
+                    help="full = the benchmark workload; medium / small = reduced cases for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -331,7 +337,8 @@ def main():
     torch.cuda.set_device(local)
     peaks, peak_src = load_peaks()
 
-    w = Workload(args.small, seed_shift=rank)
+    w = Workload(args.case, seed_shift=rank)
+    args.small = args.case != "full"
     run = Runner(w, local)
     rc = run.rc
 

@@ -8,6 +8,8 @@
 //
 //   warps 0-3  softmax of tile A      warps 4-7  softmax of tile B
 //   warp  8    TMA producer           warp  9    tcgen05.mma issuer (+ TMEM alloc)
+//   warps 10-11 idle: they complete the third warpgroup so that setmaxnreg can
+//   move registers from it to the two softmax warpgroups (128 scores per thread).
 //
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
 // S = Q K^T (both operands in 128B-swizzled shared memory, K-major); the softmax
@@ -33,7 +35,8 @@ constexpr int TILE_N = 128;
 constexpr int NSTAGE = 2;
 constexpr int BOX_BYTES = 16384;   // [128 rows][64 bf16], 128-byte swizzle
 constexpr int TILE_BYTES = 32768;  // two boxes: head_dim halves
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 384;
+constexpr int REGS_SOFTMAX = 224, REGS_AUX = 56;   // 256*224 + 128*56 = 384*168
 
 constexpr int SM_Q = 0;                              // 2 query tiles
 constexpr int SM_K = SM_Q + 2 * TILE_BYTES;          // NSTAGE key tiles
@@ -280,6 +283,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_AUX));
   if (warp == 8) {
     // ===================== TMA producer =====================
     if (lane == 0) {
@@ -370,7 +375,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       }
       __syncwarp();
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
     // ===================== softmax warpgroups =====================
     const int x = warp >> 2;                       // tile A or B
     const int row = threadIdx.x & 127;             // row of the tile = TMEM lane
@@ -431,9 +438,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
           for (int c = 0; c < 128; ++c) if (c >= lim) sr[c] = 0xff800000u;   // -inf
         }
-        float mx = __uint_as_float(sr[0]);
+        float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
 #pragma unroll
-        for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+        for (int c = 4; c < 128; c += 4) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sr[c + u]));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         const float m_new = fmaxf(m_ref, mx);
         bool need = false;
         if (i == 0) m_ref = m_new;                       // O is overwritten by the first P V
@@ -456,16 +467,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         }
         const float neg_m = -m_ref * c2;
         uint32_t pr[64];
-        float acc0 = 0.f, acc1 = 0.f;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
+        for (int c = 0; c < 64; c += 2) {
           const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), c2, neg_m));
           const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), c2, neg_m));
-          acc0 += p0; acc1 += p1;
+          const float p2 = ex2(fmaf(__uint_as_float(sr[2 * c + 2]), c2, neg_m));
+          const float p3 = ex2(fmaf(__uint_as_float(sr[2 * c + 3]), c2, neg_m));
+          acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
           pr[c] = pack2(p0, p1);
+          pr[c + 1] = pack2(p2, p3);
+          if (c == 30) TMEM_ST32(t_s + 0, pr, 0);        // first half of P goes out while the second is computed
         }
-        l_sum += acc0 + acc1;
-        TMEM_ST32(t_s + 0, pr, 0); TMEM_ST32(t_s + 32, pr, 32);
+        l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+        TMEM_ST32(t_s + 32, pr, 32);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(B_PREADY + x));
