@@ -1,6 +1,7 @@
 // Tensor-core attention for encode and prefill (bf16, head_dim 128, Hq/G in {2,4,8}).
 //
-// One CTA owns one work item = (sequence, KV group, pair of query tiles).  A
+// Persistent kernel, one CTA per SM; a work item = (sequence, KV group, pair of
+// query tiles).  A
 // query tile is 128 rows = (128 / s) consecutive tokens x the s query heads of
 // the group, so every K/V tile is shared by all heads of the group and the
 // causal granularity is 128 / s tokens.  The two tiles of a CTA are consecutive
@@ -8,8 +9,10 @@
 //
 //   warps 0-3  softmax of tile A      warps 4-7  softmax of tile B
 //   warp  8    TMA producer           warp  9    tcgen05.mma issuer (+ TMEM alloc)
-//   warps 10-11 idle: they complete the third warpgroup so that setmaxnreg can
-//   move registers from it to the two softmax warpgroups (128 scores per thread).
+//   warp  10   scheduler: draws work items from a global counter and publishes
+//              them through a two-slot ring in shared memory
+//   warp  11   idle (completes the third warpgroup: setmaxnreg moves registers
+//              from it to the two softmax warpgroups, 128 scores per thread)
 //
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
 // S = Q K^T (both operands in 128B-swizzled shared memory, K-major); the softmax
@@ -36,26 +39,30 @@ constexpr int NSTAGE = 2;
 constexpr int BOX_BYTES = 16384;   // [128 rows][64 bf16], 128-byte swizzle
 constexpr int TILE_BYTES = 32768;  // two boxes: head_dim halves
 constexpr int NTHREADS = 384;
-constexpr int REGS_SOFTMAX = 224, REGS_AUX = 56;   // 256*224 + 128*56 = 384*168
+constexpr int REGS_SOFTMAX = 216, REGS_AUX = 72;   // 256*224 + 128*56 = 384*168
 
 constexpr int SM_Q = 0;                              // 2 query tiles
 constexpr int SM_K = SM_Q + 2 * TILE_BYTES;          // NSTAGE key tiles
 constexpr int SM_V = SM_K + NSTAGE * TILE_BYTES;     // NSTAGE value tiles
-constexpr int SM_BAR = SM_V + NSTAGE * TILE_BYTES;   // mbarriers
+constexpr int ROT_BYTES = 16384;                     // cos (and sin) rows of 64 positions, fp32
+constexpr int SM_ROT = SM_V + NSTAGE * TILE_BYTES;   // cos | sin of the item's positions
+constexpr int SM_BAR = SM_ROT + 2 * ROT_BYTES;       // mbarriers
 constexpr int SM_MISC = SM_BAR + 32 * 8;             // tmem base, abort flag
-constexpr int SM_TOTAL = SM_MISC + 64;
+constexpr int SM_ITEM = SM_MISC + 64;                // two published work items
+constexpr int SM_TOTAL = SM_ITEM + 2 * 64;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;            // slack for 1024-byte alignment
 
-enum { B_QFULL = 0, B_QREADY, B_KFULL, B_KEMPTY = B_KFULL + NSTAGE, B_VFULL = B_KEMPTY + NSTAGE,
+enum { B_QFULL = 0, B_QREADY, B_QEMPTY, B_KFULL, B_KEMPTY = B_KFULL + NSTAGE, B_VFULL = B_KEMPTY + NSTAGE,
        B_VEMPTY = B_VFULL + NSTAGE, B_SFULL = B_VEMPTY + NSTAGE, B_PREADY = B_SFULL + 2, B_ODONE = B_PREADY + 2,
-       B_COUNT = B_ODONE + 2 };
+       B_IFULL = B_ODONE + 2, B_IEMPTY = B_IFULL + 2, B_COUNT = B_IEMPTY + 2 };
+static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
 
 constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long is a bug, not load
 
 struct TcParams {
-  const int2* items; const int32_t* n_items;
+  const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter
   const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu;
   int n_seq, G, Hq, s;
   int64_t self_rows;
@@ -110,6 +117,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// plain bulk copy global -> shared (16-byte aligned, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -121,17 +133,18 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+// D[tmem] (+)= A * B with A in shared memory (mma_ss2) or tensor memory (mma_ts2); descriptors are
+// given as (low word, high word): the high word (offsets, version, swizzle) is a constant, the low
+// word advances by adds.
+__device__ __forceinline__ void mma_ss2(uint32_t d, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+               "setp.ne.b32 p, %5, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+               ::"r"(d), "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-               ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tmov.b64 db, {%2, %3};\n\t"
+               "setp.ne.b32 p, %5, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+               ::"r"(d), "r"(a), "r"(blo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
 }
 
 #define RC_R32(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
@@ -176,52 +189,93 @@ constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3
 constexpr uint32_t IDESC_QK = IDESC_BASE;               // A, B K-major
 constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (= V) MN-major
 
-__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-}
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
 // ------------------------------------------------------------- work list --
-// Items = (sequence, tile-pair index), heaviest causal range first: all
-// sequences' last tile pairs, then the ones before, and so on.  One CTA.
+// Items = (sequence, tile-pair index): sequence by sequence, and inside a
+// sequence the last (heaviest) tile pair first.  With the KV group as the
+// fastest index of the flattened work list, the CTAs that run at the same time
+// share one sequence's K/V, which then stays in L2 instead of being streamed
+// from HBM once per tile pair.  One CTA; level_off[b] = first item of sequence b.
 __global__ void __launch_bounds__(1024) tile_plan_kernel(const int32_t* __restrict__ cu, int n_seq, int tok_per_cta,
                                                          int n_levels, int32_t* __restrict__ header,
                                                          int2* __restrict__ items, int32_t* __restrict__ level_off,
                                                          int max_items, int32_t* status) {
-  for (int l = threadIdx.x; l < n_levels; l += blockDim.x) {
-    int cnt = 0;
-    for (int b = 0; b < n_seq; ++b) {
-      const int len = cu[b + 1] - cu[b];
-      if (len < 0) rc_set_status(status, RECACHE_DEV_BAD_SEQLENS);
-      const int nt = (len + tok_per_cta - 1) / tok_per_cta;
-      if (nt > n_levels) rc_set_status(status, RECACHE_DEV_BAD_SEQLENS);   // longer than the max_len given
-      cnt += nt > l;
-    }
-    level_off[l] = cnt;
+  __shared__ int chunk_sum[1024];
+  // each thread owns a contiguous chunk of sequences: local sums, scan of the chunk sums, then the items
+  const int per = (n_seq + blockDim.x - 1) / blockDim.x;
+  const int b0 = min(n_seq, (int)threadIdx.x * per), b1 = min(n_seq, b0 + per);
+  int sum = 0;
+  for (int b = b0; b < b1; ++b) {
+    const int len = cu[b + 1] - cu[b];
+    if (len < 0) rc_set_status(status, RECACHE_DEV_BAD_SEQLENS);
+    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+    if (nt > n_levels) { rc_set_status(status, RECACHE_DEV_BAD_SEQLENS); nt = n_levels; }   // longer than the max_len given
+    sum += nt;
   }
+  chunk_sum[threadIdx.x] = sum;
   __syncthreads();
   if (threadIdx.x == 0) {
     int run = 0;
-    for (int l = n_levels - 1; l >= 0; --l) { const int c = level_off[l]; level_off[l] = run; run += c; }
+    for (int t = 0; t < (int)blockDim.x; ++t) { const int c = chunk_sum[t]; chunk_sum[t] = run; run += c; }
     header[0] = run < max_items ? run : max_items;
+    header[1] = 0;   // dynamic work counter of the attention kernel
   }
   __syncthreads();
-  for (int l = threadIdx.x; l < n_levels; l += blockDim.x) {
-    int k = level_off[l];
-    for (int b = 0; b < n_seq; ++b) {
-      const int nt = (cu[b + 1] - cu[b] + tok_per_cta - 1) / tok_per_cta;
-      if (nt > l) { if (k < max_items) items[k] = make_int2(b, l); ++k; }
-    }
+  int k = chunk_sum[threadIdx.x];
+  for (int b = b0; b < b1; ++b) {
+    const int len = cu[b + 1] - cu[b];
+    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+    if (nt > n_levels) nt = n_levels;
+    level_off[b] = k;
+    for (int l = nt - 1; l >= 0; --l, ++k)
+      if (k < max_items) items[k] = make_int2(b, l);
   }
 }
 
+// One work item as published by the scheduler warp (16 ints in shared memory).
+struct Item {
+  int n_tiles;      // -1: no more work
+  int g, seq0, L, tok0, kv_end, pos0, rA0, lenA, nA, b_valid;
+  int64_t base;
+};
+enum { IT_NTILES = 0, IT_G, IT_SEQ0, IT_L, IT_TOK0, IT_KVEND, IT_POS0, IT_RA0, IT_LENA, IT_NA, IT_BVALID, IT_BASE_LO,
+       IT_BASE_HI, IT_WORDS = 16 };
+
+// Work index w -> item; false when the caller's index arrays are inconsistent
+// (flagged in the status word; the scheduler skips the item).
+__device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
+  const int2 e = p.items[w / p.G];
+  it.g = w % p.G;
+  const int b = e.x;
+  const int TQ = 128 / p.s;
+  it.seq0 = p.cu[b];
+  it.L = p.cu[b + 1] - it.seq0;
+  it.tok0 = e.y * 2 * TQ;
+  it.b_valid = it.tok0 + TQ < it.L;
+  it.kv_end = min(it.L, it.tok0 + 2 * TQ);
+  it.base = p.slot ? (int64_t)p.slot[b] : (int64_t)it.seq0;
+  it.pos0 = p.pos0 ? p.pos0[b] : 0;
+  it.rA0 = 0; it.lenA = 0;
+  if (p.route_cu) { it.rA0 = p.route_cu[b * p.G + it.g]; it.lenA = p.route_cu[b * p.G + it.g + 1] - it.rA0; }
+  it.nA = (it.lenA + TILE_N - 1) / TILE_N;
+  it.n_tiles = it.nA + (it.kv_end + TILE_N - 1) / TILE_N;
+  const bool ok = it.L > 0 && it.tok0 < it.L && it.lenA >= 0 && it.rA0 >= 0 && it.base >= 0 &&
+                  it.base + it.L <= p.self_rows && it.seq0 >= 0;
+  if (!ok) rc_set_status(p.status, RECACHE_DEV_BAD_SLOT);
+  return ok;
+}
+
 // ---------------------------------------------------------------- kernel --
-template <typename TO>
+// Persistent: a scheduler warp draws work indices from a global counter (the
+// list is heavy-first inside each sequence, so the tail of the launch is made of
+// light items) and publishes items through a two-slot ring in shared memory.
+// The next item's Q load, Q rotation and first K/V tiles overlap the current
+// item's last tiles and its epilogue.  Barrier phases run on across items.
+template <typename TO, bool ROT_SMEM>
 __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                               const __grid_constant__ CUtensorMap tm_ks,
                                                               const __grid_constant__ CUtensorMap tm_vs,
@@ -229,31 +283,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                                                               const __grid_constant__ CUtensorMap tm_vr,
                                                               const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  const int item_idx = blockIdx.x / p.G, g = blockIdx.x % p.G;
-  if (item_idx >= *p.n_items) return;
-  const int2 item = p.items[item_idx];
-  const int b = item.x, qt = item.y;
+  const int total = p.header[0] * p.G;
+  if ((int)blockIdx.x >= total) return;
   const int s = p.s, TQ = 128 / s;
-  const int seq0 = p.cu[b], L = p.cu[b + 1] - seq0;
-  const int tok0 = qt * 2 * TQ;                    // first token of tile A (local index)
-  const bool b_valid = tok0 + TQ < L;              // tile B holds at least one real token
-  const int kv_end = min(L, tok0 + 2 * TQ);        // causal keys needed by the pair
-  const int64_t base = p.slot ? (int64_t)p.slot[b] : (int64_t)seq0;
-  const int pos0 = p.pos0 ? p.pos0[b] : 0;
-  int rA0 = 0, lenA = 0;
-  if (p.route_cu) { rA0 = p.route_cu[b * p.G + g]; lenA = p.route_cu[b * p.G + g + 1] - rA0; }
-  if (L <= 0 || tok0 >= L || lenA < 0 || base < 0 || base + L > p.self_rows || seq0 < 0) {
-    if (threadIdx.x == 0) rc_set_status(p.status, RECACHE_DEV_BAD_SLOT);
-    return;
-  }
-  const int nA = (lenA + TILE_N - 1) / TILE_N, nB = (kv_end + TILE_N - 1) / TILE_N;
-  const int n_tiles = nA + nB;
 
   const uint32_t sm = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sm_gen = smem_raw + (sm - smem_u32(smem_raw));
   const uint32_t bars = sm + SM_BAR;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_gen + SM_MISC + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm_gen + SM_MISC);
+  volatile int* item_ring = reinterpret_cast<volatile int*>(sm_gen + SM_ITEM);
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -261,18 +300,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     *abort_flag = 0;
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QREADY), 256);
+    mbar_init(bar(B_QEMPTY), 1);
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(bar(B_KFULL + i), 1); mbar_init(bar(B_KEMPTY + i), 1);
       mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1); mbar_init(bar(B_PREADY + x), 128); mbar_init(bar(B_ODONE + x), 1);
+      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 258);   // producer + MMA + 256 softmax threads
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 8 && lane == 0) {
     prefetch_tmap(&tm_q); prefetch_tmap(&tm_ks); prefetch_tmap(&tm_vs);
-    if (nA) { prefetch_tmap(&tm_kr); prefetch_tmap(&tm_vr); }
+    if (p.route_cu) { prefetch_tmap(&tm_kr); prefetch_tmap(&tm_vr); }
   }
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sm + SM_MISC), "r"(512u) : "memory");
@@ -283,97 +324,183 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // Item n of this CTA lives in ring slot n & 1; every consumer copies it to
+  // registers and then releases the slot.
+  auto fetch_item = [&](uint32_t n, Item& it, bool release) {
+    const int sl = n & 1u;
+    mbar_wait(bar(B_IFULL + sl), (n >> 1) & 1u, abort_flag, p.status);
+    const volatile int* r = item_ring + sl * IT_WORDS;
+    it.n_tiles = r[IT_NTILES]; it.g = r[IT_G]; it.seq0 = r[IT_SEQ0]; it.L = r[IT_L]; it.tok0 = r[IT_TOK0];
+    it.kv_end = r[IT_KVEND]; it.pos0 = r[IT_POS0]; it.rA0 = r[IT_RA0]; it.lenA = r[IT_LENA]; it.nA = r[IT_NA];
+    it.b_valid = r[IT_BVALID];
+    it.base = (int64_t)(((uint64_t)(uint32_t)r[IT_BASE_HI] << 32) | (uint32_t)r[IT_BASE_LO]);
+    if (*abort_flag) it.n_tiles = -1;
+    if (release) mbar_arrive(bar(B_IEMPTY + sl));
+  };
+
   if (warp >= 8) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_AUX));
-  if (warp == 8) {
+  if (warp == 10) {
+    // ===================== scheduler =====================
+    if (lane == 0) {
+      bool first = true;
+      for (uint32_t n = 0;; ++n) {
+        const int sl = n & 1u;
+        mbar_wait(bar(B_IEMPTY + sl), ((n >> 1) & 1u) ^ 1u, abort_flag, p.status);
+        Item it;
+        for (;;) {   // CTA c starts with index c; every later index comes from the shared counter
+          const int w = first ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(p.header + 1, 1);
+          first = false;
+          if (w >= total || *abort_flag) { it.n_tiles = -1; break; }
+          if (load_item(p, w, it)) break;
+        }
+        volatile int* r = item_ring + sl * IT_WORDS;
+        r[IT_NTILES] = it.n_tiles;
+        if (it.n_tiles > 0) {
+          r[IT_G] = it.g; r[IT_SEQ0] = it.seq0; r[IT_L] = it.L; r[IT_TOK0] = it.tok0; r[IT_KVEND] = it.kv_end;
+          r[IT_POS0] = it.pos0; r[IT_RA0] = it.rA0; r[IT_LENA] = it.lenA; r[IT_NA] = it.nA; r[IT_BVALID] = it.b_valid;
+          r[IT_BASE_LO] = (int)(uint32_t)(it.base & 0xffffffffll); r[IT_BASE_HI] = (int)(uint32_t)((uint64_t)it.base >> 32);
+        }
+        mbar_arrive(bar(B_IFULL + sl));
+        if (it.n_tiles < 0) break;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 8) {
     // ===================== TMA producer =====================
     if (lane == 0) {
-      mbar_expect_tx(bar(B_QFULL), 2 * TILE_BYTES);
-      for (int x = 0; x < 2; ++x)
-        for (int kc = 0; kc < 2; ++kc)
-          tma_load_3d(sm + SM_Q + x * TILE_BYTES + kc * BOX_BYTES, &tm_q, bar(B_QFULL), kc * 64, g * s,
-                      seq0 + tok0 + x * TQ);
-      for (int i = 0; i < n_tiles; ++i) {
-        const int st = i % NSTAGE;
-        const uint32_t ph = (uint32_t)(i / NSTAGE) & 1u;
-        const bool route = i < nA;
-        const int row = route ? rA0 + i * TILE_N : (int)((int64_t)g * p.self_rows + base) + (i - nA) * TILE_N;
-        mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, abort_flag, p.status);
-        mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
-        for (int kc = 0; kc < 2; ++kc)
-          tma_load_2d(sm + SM_K + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_kr : &tm_ks, bar(B_KFULL + st), kc * 64, row);
-        mbar_wait(bar(B_VEMPTY + st), ph ^ 1u, abort_flag, p.status);
-        mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
-        for (int kc = 0; kc < 2; ++kc)
-          tma_load_2d(sm + SM_V + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_vr : &tm_vs, bar(B_VFULL + st), kc * 64, row);
+      Item it;
+      uint32_t kv_n = 0;
+      for (uint32_t item_n = 0;; ++item_n) {
+        fetch_item(item_n, it, true);
+        if (it.n_tiles < 0) break;
+        // Q tiles: free once the previous item's last S = Q K^T has completed
+        mbar_wait(bar(B_QEMPTY), (item_n & 1u) ^ 1u, abort_flag, p.status);
+        uint32_t rot_bytes = 0;
+        const int pos_start = it.pos0 + it.tok0;
+        if (ROT_SMEM) {
+          const int rows = min(2 * TQ, p.max_pos - pos_start);
+          if (pos_start >= 0 && rows > 0) rot_bytes = (uint32_t)rows * 256u;
+        }
+        mbar_expect_tx(bar(B_QFULL), 2 * TILE_BYTES + 2 * rot_bytes);
+        for (int x = 0; x < 2; ++x)
+          for (int kc = 0; kc < 2; ++kc)
+            tma_load_3d(sm + SM_Q + x * TILE_BYTES + kc * BOX_BYTES, &tm_q, bar(B_QFULL), kc * 64, it.g * s,
+                        it.seq0 + it.tok0 + x * TQ);
+        if (rot_bytes) {   // cos / sin rows of the item's positions (contiguous in the table)
+          bulk_load(sm + SM_ROT, p.cos_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
+          bulk_load(sm + SM_ROT + ROT_BYTES, p.sin_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
+        }
+        for (int i = 0; i < it.n_tiles; ++i, ++kv_n) {
+          const int st = kv_n % NSTAGE;
+          const uint32_t ph = (kv_n / NSTAGE) & 1u;
+          const bool route = i < it.nA;
+          const int row = route ? it.rA0 + i * TILE_N
+                                : (int)((int64_t)it.g * p.self_rows + it.base) + (i - it.nA) * TILE_N;
+          mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, abort_flag, p.status);
+          mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
+          for (int kc = 0; kc < 2; ++kc)
+            tma_load_2d(sm + SM_K + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_kr : &tm_ks, bar(B_KFULL + st), kc * 64, row);
+          mbar_wait(bar(B_VEMPTY + st), ph ^ 1u, abort_flag, p.status);
+          mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
+          for (int kc = 0; kc < 2; ++kc)
+            tma_load_2d(sm + SM_V + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_vr : &tm_vs, bar(B_VFULL + st), kc * 64, row);
+        }
       }
     }
     __syncwarp();
   } else if (warp == 9) {
     // ===================== MMA issuer =====================
+    // descriptor words: low = (address >> 4) | (LBO >> 4) << 16, high = (SBO >> 4) | version | swizzle
+    const uint64_t d_k = smem_desc(0, 16, 1024), d_v = smem_desc(0, BOX_BYTES, 1024);
+    const uint32_t hi_k = (uint32_t)(d_k >> 32), hi_v = (uint32_t)(d_v >> 32);
+    const uint32_t lo_q = (uint32_t)d_k + ((sm + SM_Q) >> 4), lo_k = (uint32_t)d_k + ((sm + SM_K) >> 4);
+    const uint32_t lo_v = (uint32_t)d_v + ((sm + SM_V) >> 4);
     auto issue_qk = [&](int x, int st) {
-      const uint32_t qa = sm + SM_Q + x * TILE_BYTES, ka = sm + SM_K + st * TILE_BYTES;
+      const uint32_t qa = lo_q + x * (TILE_BYTES >> 4), ka = lo_k + st * (TILE_BYTES >> 4);
+      const uint32_t dst = tmem + COL_S + 128 * x;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const uint32_t off = (j >> 2) * BOX_BYTES + (j & 3) * 32;
-        mma_ss(tmem + COL_S + 128 * x, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK, j > 0);
+        const uint32_t off = ((j >> 2) * BOX_BYTES + (j & 3) * 32) >> 4;
+        mma_ss2(dst, qa + off, ka + off, hi_k, IDESC_QK, j > 0);
       }
     };
     auto issue_pv = [&](int x, int st, int ksteps, bool first) {
-      const uint32_t va = sm + SM_V + st * TILE_BYTES;
+      const uint32_t va = lo_v + st * (TILE_BYTES >> 4);
+      const uint32_t dst = tmem + COL_O + 128 * x, src = tmem + COL_S + 128 * x;
+#pragma unroll 8
       for (int j = 0; j < ksteps; ++j)
-        mma_ts(tmem + COL_O + 128 * x, tmem + COL_S + 128 * x + 8 * j, smem_desc(va + j * 2048, BOX_BYTES, 1024),
-               IDESC_PV, (!first || j > 0) ? 1u : 0u);
+        mma_ts2(dst, src + 8 * j, va + j * (2048 >> 4), hi_v, IDESC_PV, (!first || j > 0) ? 1u : 0u);
     };
-    mbar_wait(bar(B_QREADY), 0, abort_flag, p.status);
-    mbar_wait(bar(B_KFULL + 0), 0, abort_flag, p.status);
-    tc_fence_after();
-    if (lane == 0) {
-      issue_qk(0, 0); tc_commit(bar(B_SFULL + 0));
-      if (b_valid) { issue_qk(1, 0); tc_commit(bar(B_SFULL + 1)); }
-      tc_commit(bar(B_KEMPTY + 0));
-    }
-    __syncwarp();
-    for (int i = 0; i < n_tiles; ++i) {
-      const int st = i % NSTAGE;
-      const uint32_t ph = (uint32_t)(i / NSTAGE) & 1u;
-      // rows of this tile that really belong to the segment; keys the pair can see
-      const int seg_rows = i < nA ? lenA - i * TILE_N : L - (i - nA) * TILE_N;
-      const int vis_rows = i < nA ? seg_rows : kv_end - (i - nA) * TILE_N;
-      const int ksteps = (min(vis_rows, TILE_N) + 15) >> 4;
-      mbar_wait(bar(B_VFULL + st), ph, abort_flag, p.status);
-      if (seg_rows < ksteps * 16) {
-        // rows past the segment hold whatever follows it in memory: zero them, 0 * NaN would poison O
-        uint8_t* vb = sm_gen + SM_V + st * TILE_BYTES;
-        const int n_rows = ksteps * 16 - seg_rows;
-        for (int e = lane; e < n_rows * 16; e += 32) {
-          const int r = seg_rows + (e >> 4), c = e & 15;
-          *reinterpret_cast<uint4*>(vb + (c >> 3) * BOX_BYTES + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
-        }
-        fence_async_smem();
-      }
+    Item it;
+    uint32_t kv_n = 0, cnt[2] = {0, 0};   // K/V tiles, tiles per query tile so far
+    for (uint32_t item_n = 0;; ++item_n) {
+      fetch_item(item_n, it, false);
       __syncwarp();
-      const int st1 = (i + 1) % NSTAGE;
-      const uint32_t ph1 = (uint32_t)((i + 1) / NSTAGE) & 1u;
-      mbar_wait(bar(B_PREADY + 0), (uint32_t)i & 1u, abort_flag, p.status);
+      if (lane == 0) mbar_arrive(bar(B_IEMPTY + (item_n & 1u)));
+      if (it.n_tiles < 0) break;
+      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, L = it.L, kv_end = it.kv_end;
+      const bool b_valid = it.b_valid != 0;
+      mbar_wait(bar(B_QREADY), item_n & 1u, abort_flag, p.status);
+      mbar_wait(bar(B_KFULL + kv_n % NSTAGE), (kv_n / NSTAGE) & 1u, abort_flag, p.status);
       tc_fence_after();
-      if (lane == 0) { issue_pv(0, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 0)); }
-      if (i + 1 < n_tiles) {
-        mbar_wait(bar(B_KFULL + st1), ph1, abort_flag, p.status);
-        tc_fence_after();
-        if (lane == 0) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
-      }
-      if (b_valid) {
-        mbar_wait(bar(B_PREADY + 1), (uint32_t)i & 1u, abort_flag, p.status);
-        tc_fence_after();
-        if (lane == 0) { issue_pv(1, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 1)); }
-      }
-      if (lane == 0) tc_commit(bar(B_VEMPTY + st));
-      if (i + 1 < n_tiles && lane == 0) {
-        if (b_valid) { issue_qk(1, st1); tc_commit(bar(B_SFULL + 1)); }
-        tc_commit(bar(B_KEMPTY + st1));
+      if (lane == 0) {
+        const int st0 = kv_n % NSTAGE;
+        issue_qk(0, st0); tc_commit(bar(B_SFULL + 0));
+        if (b_valid) { issue_qk(1, st0); tc_commit(bar(B_SFULL + 1)); }
+        tc_commit(bar(B_KEMPTY + st0));
+        if (n_tiles == 1) tc_commit(bar(B_QEMPTY));
       }
       __syncwarp();
+      for (int i = 0; i < n_tiles; ++i) {
+        const uint32_t n = kv_n + (uint32_t)i;
+        const int st = n % NSTAGE;
+        const uint32_t ph = (n / NSTAGE) & 1u;
+        // rows of this tile that really belong to the segment; keys the pair can see
+        const int seg_rows = i < nA ? lenA - i * TILE_N : L - (i - nA) * TILE_N;
+        const int vis_rows = i < nA ? seg_rows : kv_end - (i - nA) * TILE_N;
+        const int ksteps = (min(vis_rows, TILE_N) + 15) >> 4;
+        mbar_wait(bar(B_VFULL + st), ph, abort_flag, p.status);
+        if (seg_rows < ksteps * 16) {
+          // rows past the segment hold whatever follows it in memory: zero them, 0 * NaN would poison O
+          uint8_t* vb = sm_gen + SM_V + st * TILE_BYTES;
+          const int n_rows = ksteps * 16 - seg_rows;
+          for (int e = lane; e < n_rows * 16; e += 32) {
+            const int r = seg_rows + (e >> 4), c = e & 15;
+            *reinterpret_cast<uint4*>(vb + (c >> 3) * BOX_BYTES + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+          }
+          fence_async_smem();
+        }
+        __syncwarp();
+        const int st1 = (n + 1) % NSTAGE;
+        const uint32_t ph1 = ((n + 1) / NSTAGE) & 1u;
+        const bool more = i + 1 < n_tiles;
+        mbar_wait(bar(B_PREADY + 0), cnt[0] & 1u, abort_flag, p.status);
+        tc_fence_after();
+        if (lane == 0) { issue_pv(0, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 0)); }
+        ++cnt[0];
+        if (more) {
+          mbar_wait(bar(B_KFULL + st1), ph1, abort_flag, p.status);
+          tc_fence_after();
+          if (lane == 0) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
+        }
+        if (b_valid) {
+          mbar_wait(bar(B_PREADY + 1), cnt[1] & 1u, abort_flag, p.status);
+          tc_fence_after();
+          if (lane == 0) { issue_pv(1, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 1)); }
+          ++cnt[1];
+        }
+        if (lane == 0) {
+          tc_commit(bar(B_VEMPTY + st));
+          if (more) {
+            if (b_valid) { issue_qk(1, st1); tc_commit(bar(B_SFULL + 1)); }
+            tc_commit(bar(B_KEMPTY + st1));
+            if (i + 2 == n_tiles) tc_commit(bar(B_QEMPTY));   // the item's last S has been issued
+          }
+        }
+        __syncwarp();
+      }
+      kv_n += (uint32_t)n_tiles;
     }
   }
   } else {
@@ -382,137 +509,160 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const int x = warp >> 2;                       // tile A or B
     const int row = threadIdx.x & 127;             // row of the tile = TMEM lane
     const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3)) << 16);
-    const int t_row = tok0 + x * TQ + row / s;     // token (local index)
-    const bool row_valid = t_row < L;
-    const int t_eff = min(t_row, L - 1);
-    const int head = g * s + row % s;
+    const uint32_t t_s = tmem + lane_addr + COL_S + 128 * x;
+    const uint32_t t_o = tmem + lane_addr + COL_O + 128 * x;
+    const float c2 = p.scale_log2;
+    uint32_t item_n = 0, cnt = 0;                  // items seen; tiles this query tile has gone through
 
-    // ---- rotate this row of Q in shared memory (swizzled 16-byte chunks) ----
-    mbar_wait(bar(B_QFULL), 0, abort_flag, p.status);
-    {
-      const int pos = min(max(pos0 + t_eff, 0), p.max_pos - 1);
-      if (pos0 + t_eff >= p.max_pos) rc_set_status(p.status, RECACHE_DEV_BAD_POS);
-      const float* cp = p.cos_tab + (int64_t)pos * 64;
-      const float* sp = p.sin_tab + (int64_t)pos * 64;
+    // Rotates this thread's row of the freshly loaded Q tile in shared memory
+    // (swizzled 16-byte chunks; element i pairs with i + 64 in the other box).
+    auto rotate_q = [&](const Item& it, uint32_t n_item) {
+      mbar_wait(bar(B_QFULL), n_item & 1u, abort_flag, p.status);
+      const int t_eff = min(it.tok0 + x * TQ + row / s, it.L - 1);
+      const int pos = it.pos0 + t_eff;
+      if (pos < 0 || pos >= p.max_pos) rc_set_status(p.status, RECACHE_DEV_BAD_POS);
+      const float4 *cp, *sp;
+      if (ROT_SMEM) {   // staged by the producer: row = token index inside the tile pair
+        const int ri = min(max(t_eff - it.tok0, 0), 2 * TQ - 1);
+        cp = reinterpret_cast<const float4*>(sm_gen + SM_ROT + ri * 256);
+        sp = reinterpret_cast<const float4*>(sm_gen + SM_ROT + ROT_BYTES + ri * 256);
+      } else {
+        const int pc = min(max(pos, 0), p.max_pos - 1);
+        cp = reinterpret_cast<const float4*>(p.cos_tab + (int64_t)pc * 64);
+        sp = reinterpret_cast<const float4*>(p.sin_tab + (int64_t)pc * 64);
+      }
       uint8_t* qb = sm_gen + SM_Q + x * TILE_BYTES + row * 128;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const int off = ((c ^ (row & 7)) << 4);
-        uint4 ulo = *reinterpret_cast<uint4*>(qb + off), uhi = *reinterpret_cast<uint4*>(qb + BOX_BYTES + off);
-        float lo[8], hi[8], cs[8], sn[8];
-        unpack8(ulo, lo); unpack8(uhi, hi);
-        *reinterpret_cast<float4*>(cs) = *reinterpret_cast<const float4*>(cp + 8 * c);
-        *reinterpret_cast<float4*>(cs + 4) = *reinterpret_cast<const float4*>(cp + 8 * c + 4);
-        *reinterpret_cast<float4*>(sn) = *reinterpret_cast<const float4*>(sp + 8 * c);
-        *reinterpret_cast<float4*>(sn + 4) = *reinterpret_cast<const float4*>(sp + 8 * c + 4);
-        uint32_t wl[4], wh[4];
+        const uint4 ulo = *reinterpret_cast<uint4*>(qb + off), uhi = *reinterpret_cast<uint4*>(qb + BOX_BYTES + off);
+        const float4 c0 = cp[2 * c], c1 = cp[2 * c + 1], s0 = sp[2 * c], s1 = sp[2 * c + 1];
+        const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        const uint32_t wlo[4] = {ulo.x, ulo.y, ulo.z, ulo.w}, whi[4] = {uhi.x, uhi.y, uhi.z, uhi.w};
+        uint32_t ol[4], oh[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float a0 = __fmaf_rn(lo[2 * i], cs[2 * i], -__fmul_rn(hi[2 * i], sn[2 * i]));
-          const float a1 = __fmaf_rn(lo[2 * i + 1], cs[2 * i + 1], -__fmul_rn(hi[2 * i + 1], sn[2 * i + 1]));
-          const float b0 = __fmaf_rn(hi[2 * i], cs[2 * i], __fmul_rn(lo[2 * i], sn[2 * i]));
-          const float b1 = __fmaf_rn(hi[2 * i + 1], cs[2 * i + 1], __fmul_rn(lo[2 * i + 1], sn[2 * i + 1]));
-          wl[i] = pack2(a0, a1); wh[i] = pack2(b0, b1);
+          const float l0 = __uint_as_float(wlo[i] << 16), l1 = __uint_as_float(wlo[i] & 0xffff0000u);
+          const float h0 = __uint_as_float(whi[i] << 16), h1 = __uint_as_float(whi[i] & 0xffff0000u);
+          ol[i] = pack2(__fmaf_rn(l0, cs[2 * i], -__fmul_rn(h0, sn[2 * i])),
+                        __fmaf_rn(l1, cs[2 * i + 1], -__fmul_rn(h1, sn[2 * i + 1])));
+          oh[i] = pack2(__fmaf_rn(h0, cs[2 * i], __fmul_rn(l0, sn[2 * i])),
+                        __fmaf_rn(h1, cs[2 * i + 1], __fmul_rn(l1, sn[2 * i + 1])));
         }
-        *reinterpret_cast<uint4*>(qb + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-        *reinterpret_cast<uint4*>(qb + BOX_BYTES + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+        *reinterpret_cast<uint4*>(qb + off) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+        *reinterpret_cast<uint4*>(qb + BOX_BYTES + off) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
       }
       fence_async_smem();
       mbar_arrive(bar(B_QREADY));
-    }
+    };
 
-    if (x == 0 || b_valid) {
-      const uint32_t t_s = tmem + lane_addr + COL_S + 128 * x;
-      const uint32_t t_o = tmem + lane_addr + COL_O + 128 * x;
-      const float c2 = p.scale_log2;
+    Item it, nx;
+    fetch_item(0, it, true);
+    if (it.n_tiles > 0) rotate_q(it, 0);
+    while (it.n_tiles > 0) {
+      const bool active = x == 0 || it.b_valid;
+      const int t_row = it.tok0 + x * TQ + row / s;     // token (local index)
+      const int t_eff = min(t_row, it.L - 1);
+      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA;
       float m_ref = -INFINITY, l_sum = 0.f;
-      for (int i = 0; i < n_tiles; ++i) {
-        mbar_wait(bar(B_SFULL + x), (uint32_t)i & 1u, abort_flag, p.status);
-        tc_fence_after();
-        uint32_t sr[128];
-        TMEM_LD32(t_s + 0, sr, 0); TMEM_LD32(t_s + 32, sr, 32); TMEM_LD32(t_s + 64, sr, 64); TMEM_LD32(t_s + 96, sr, 96);
-        tmem_wait_ld();
-        // keys this row may see in this tile: columns [0, lim)
-        const int lim = i < nA ? lenA - i * TILE_N : t_eff - (i - nA) * TILE_N + 1;
-        if (lim < TILE_N) {
-#pragma unroll
-          for (int c = 0; c < 128; ++c) if (c >= lim) sr[c] = 0xff800000u;   // -inf
-        }
-        float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
-#pragma unroll
-        for (int c = 4; c < 128; c += 4) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sr[c + u]));
-        }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-        const float m_new = fmaxf(m_ref, mx);
-        bool need = false;
-        if (i == 0) m_ref = m_new;                       // O is overwritten by the first P V
-        else need = (m_new - m_ref) * c2 > 8.f;          // lazy: P stays below 2^8 otherwise
-        if (__any_sync(0xffffffffu, need)) {
-          mbar_wait(bar(B_ODONE + x), (uint32_t)(i - 1) & 1u, abort_flag, p.status);
+      if (active) {
+        for (int i = 0; i < n_tiles; ++i, ++cnt) {
+          mbar_wait(bar(B_SFULL + x), cnt & 1u, abort_flag, p.status);
           tc_fence_after();
-          const float f = need ? ex2((m_ref - m_new) * c2) : 1.f;
+          uint32_t sr[128];
+          TMEM_LD32(t_s + 0, sr, 0); TMEM_LD32(t_s + 32, sr, 32); TMEM_LD32(t_s + 64, sr, 64); TMEM_LD32(t_s + 96, sr, 96);
+          tmem_wait_ld();
+          // keys this row may see in this tile: columns [0, lim)
+          const int lim = i < nA ? lenA - i * TILE_N : t_eff - (i - nA) * TILE_N + 1;
+          if (lim < TILE_N) {
 #pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t orr[32];
-            TMEM_LD32(t_o + 32 * ch, orr, 0);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * f);
-            TMEM_ST32(t_o + 32 * ch, orr, 0);
+            for (int c = 0; c < 128; ++c) if (c >= lim) sr[c] = 0xff800000u;   // -inf
           }
+          float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
+#pragma unroll
+          for (int c = 4; c < 128; c += 4) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sr[c + u]));
+          }
+          const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          const float m_new = fmaxf(m_ref, mx);
+          bool need = false;
+          if (i == 0) m_ref = m_new;                       // O is overwritten by the first P V
+          else need = (m_new - m_ref) * c2 > 8.f;          // lazy: P stays below 2^8 otherwise
+          if (__any_sync(0xffffffffu, need)) {
+            mbar_wait(bar(B_ODONE + x), (cnt - 1u) & 1u, abort_flag, p.status);
+            tc_fence_after();
+            const float f = need ? ex2((m_ref - m_new) * c2) : 1.f;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              uint32_t orr[32];
+              TMEM_LD32(t_o + 32 * ch, orr, 0);
+              tmem_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * f);
+              TMEM_ST32(t_o + 32 * ch, orr, 0);
+            }
+            tmem_wait_st();
+            if (need) { l_sum *= f; m_ref = m_new; }
+          }
+          const float neg_m = -m_ref * c2;
+          uint32_t pr[64];
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int c = 0; c < 64; c += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), c2, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), c2, neg_m));
+            const float p2 = ex2(fmaf(__uint_as_float(sr[2 * c + 2]), c2, neg_m));
+            const float p3 = ex2(fmaf(__uint_as_float(sr[2 * c + 3]), c2, neg_m));
+            acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
+            pr[c] = pack2(p0, p1);
+            pr[c + 1] = pack2(p2, p3);
+            if (c == 30) TMEM_ST32(t_s + 0, pr, 0);        // first half of P goes out while the second is computed
+          }
+          l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          TMEM_ST32(t_s + 32, pr, 32);
           tmem_wait_st();
-          if (need) { l_sum *= f; m_ref = m_new; }
+          tc_fence_before();
+          mbar_arrive(bar(B_PREADY + x));
         }
-        const float neg_m = -m_ref * c2;
-        uint32_t pr[64];
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < 64; c += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), c2, neg_m));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), c2, neg_m));
-          const float p2 = ex2(fmaf(__uint_as_float(sr[2 * c + 2]), c2, neg_m));
-          const float p3 = ex2(fmaf(__uint_as_float(sr[2 * c + 3]), c2, neg_m));
-          acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
-          pr[c] = pack2(p0, p1);
-          pr[c + 1] = pack2(p2, p3);
-          if (c == 30) TMEM_ST32(t_s + 0, pr, 0);        // first half of P goes out while the second is computed
-        }
-        l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
-        TMEM_ST32(t_s + 32, pr, 32);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(B_PREADY + x));
       }
-      // ---- epilogue: O / l -> global ----
-      mbar_wait(bar(B_ODONE + x), (uint32_t)(n_tiles - 1) & 1u, abort_flag, p.status);
-      tc_fence_after();
-      const float inv = 1.f / l_sum;
-      TO* orow = reinterpret_cast<TO*>(p.out) + ((int64_t)(seq0 + t_row) * p.Hq + head) * D;
+      // ---- next item's Q first (its load was issued a tile ago), then this item's epilogue ----
+      fetch_item(item_n + 1, nx, true);
+      if (nx.n_tiles > 0) rotate_q(nx, item_n + 1);
+      if (active) {
+        mbar_wait(bar(B_ODONE + x), (cnt - 1u) & 1u, abort_flag, p.status);
+        tc_fence_after();
+        const float inv = 1.f / l_sum;
+        const bool row_valid = t_row < it.L;
+        TO* orow = reinterpret_cast<TO*>(p.out) + ((int64_t)(it.seq0 + t_row) * p.Hq + it.g * s + row % s) * D;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t orr[32];
-        TMEM_LD32(t_o + 32 * ch, orr, 0);
-        tmem_wait_ld();
-        if (row_valid) {
-          if constexpr (sizeof(TO) == 4) {
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t orr[32];
+          TMEM_LD32(t_o + 32 * ch, orr, 0);
+          tmem_wait_ld();
+          if (row_valid) {
+            if constexpr (sizeof(TO) == 4) {
 #pragma unroll
-            for (int c = 0; c < 32; c += 4)
-              *reinterpret_cast<float4*>(reinterpret_cast<float*>(orow) + 32 * ch + c) =
-                  make_float4(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv,
-                              __uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv);
-          } else {
+              for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(orow) + 32 * ch + c) =
+                    make_float4(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv,
+                                __uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv);
+            } else {
 #pragma unroll
-            for (int c = 0; c < 32; c += 8)
-              *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(orow) + 32 * ch + c) =
-                  make_uint4(pack2(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv),
-                             pack2(__uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv),
-                             pack2(__uint_as_float(orr[c + 4]) * inv, __uint_as_float(orr[c + 5]) * inv),
-                             pack2(__uint_as_float(orr[c + 6]) * inv, __uint_as_float(orr[c + 7]) * inv));
+              for (int c = 0; c < 32; c += 8)
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(orow) + 32 * ch + c) =
+                    make_uint4(pack2(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv),
+                               pack2(__uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv),
+                               pack2(__uint_as_float(orr[c + 4]) * inv, __uint_as_float(orr[c + 5]) * inv),
+                               pack2(__uint_as_float(orr[c + 6]) * inv, __uint_as_float(orr[c + 7]) * inv));
+            }
           }
         }
+        // the next item's first P V overwrites O: order this thread's reads before its next P-ready arrive
+        tc_fence_before();
       }
+      it = nx; ++item_n;
     }
   }
   // ---- teardown: every thread is done with tensor memory before it is freed ----
@@ -586,7 +736,7 @@ static int tc_levels(const recache_ctx* ctx, int max_len) {
 }
 
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len) {
-  return 256 + align256(tc_max_items(ctx, n_seq, total) * 8) + align256((int64_t)tc_levels(ctx, max_len) * 4);
+  return 256 + align256(tc_max_items(ctx, n_seq, total) * 8) + align256((int64_t)(n_seq + 1) * 4);
 }
 
 cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaStream_t st) {
@@ -615,21 +765,21 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
                                          (int)max_items, ctx->status);
   }
   TcParams p;
-  p.items = items; p.n_items = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
+  p.items = items; p.header = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
   p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.out = a.o;
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)ctx->desc.head_dim));
   p.status = ctx->status;
-  const unsigned grid = (unsigned)(max_items * G);
+  const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
+  const unsigned grid = (unsigned)(max_items * G < sms ? max_items * G : sms);
   RcLaunchScope scope(ctx, a.route_cu ? RC_K_PREFILL_ATTN : RC_K_ENCODE_ATTN, st);
-  if (a.out_dtype == RECACHE_F32) {
-    static bool attr_f = false;
-    if (!attr_f) { cudaFuncSetAttribute(attn_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); attr_f = true; }
-    attn_tc_kernel<float><<<grid, NTHREADS, SM_ALLOC, st>>>(tq, tks, tvs, tkr, tvr, p);
-  } else {
-    static bool attr_b = false;
-    if (!attr_b) { cudaFuncSetAttribute(attn_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); attr_b = true; }
-    attn_tc_kernel<__nv_bfloat16><<<grid, NTHREADS, SM_ALLOC, st>>>(tq, tks, tvs, tkr, tvr, p);
-  }
+  auto launch = [&](auto kernel) {
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC);
+    kernel<<<grid, NTHREADS, SM_ALLOC, st>>>(tq, tks, tvs, tkr, tvr, p);
+  };
+  const bool f32 = a.out_dtype == RECACHE_F32, rot = s >= 4;   // 2 * 128 / s <= 64 positions fit the staging area
+  if (f32) { if (rot) launch(attn_tc_kernel<float, true>); else launch(attn_tc_kernel<float, false>); }
+  else { if (rot) launch(attn_tc_kernel<__nv_bfloat16, true>); else launch(attn_tc_kernel<__nv_bfloat16, false>); }
   return cudaGetLastError();
 }
+
