@@ -308,6 +308,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ multi-rank --
+def max_over_ranks(ms: float, device: str = "cuda") -> float:
+    """Replica timing: every rank ran its own copy of the step; the job's time is the slowest rank's."""
+    import torch.distributed as td
+    if not (td.is_available() and td.is_initialized()) or td.get_world_size() == 1:
+        return ms
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    td.all_reduce(t, op=td.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, flops_per_rank: float, ms_step: float) -> float:
+    """Whole-job throughput (TFLOP/s): the work of all replicas over the slowest rank's time."""
+    return world * flops_per_rank / (ms_step * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------ main --
 def main():
     ap = argparse.ArgumentParser()
@@ -365,10 +381,7 @@ def main():
         kt = rc.kernel_times() if with_timer else None
         if with_timer:
             rc.kernel_timer(False)
-        if dist:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            td.all_reduce(t, op=td.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ms)
         return ms, kt, clocks
 
     ms, kt, clocks = timed(run.step, args.steps, with_timer=True)
@@ -376,12 +389,12 @@ def main():
     if code != 0:
         raise SystemExit(f"device status {code} after the timed region")
     ms_step = ms / args.steps
-    value = world * w.total_flops / (ms_step * 1e-3) / 1e12
+    value = job_value(world, w.total_flops, ms_step)
 
     e2e = None
     if not args.no_e2e:
         ms_e, _, _ = timed(run.step_e2e, args.steps)
-        e2e = {"value": world * w.total_flops / (ms_e / args.steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+        e2e = {"value": job_value(world, w.total_flops, ms_e / args.steps), "unit": "TFLOP/s",
                "ms_per_step": ms_e / args.steps, "h2d_bytes_per_step": run.h2d_bytes,
                "d2h_bytes_per_step": run.d2h_bytes}
 

@@ -121,8 +121,8 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
 def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int]],
                 storage: Optional[str] = None):
     """The same definition for a chosen set of output rows (token, head) only,
-    one at a time; for sizes where the full table takes minutes."""
-    q = np.asarray(q, F64)
+    one at a time; for sizes where the full table takes minutes.  q/k/v may be
+    fp32 arrays holding bf16 values: only the rows a sample needs are widened."""
     t, hq, d = q.shape
     g = k.shape[1]
     s = hq // g
@@ -253,7 +253,7 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
 def prefill_rows(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta: float,
                  out_rows: Sequence[Tuple[int, int]], storage: Optional[str] = None):
     """attend_prefill for chosen (query token, head) rows only."""
-    q = np.asarray(q); cu = np.asarray(cu_q)
+    cu = np.asarray(cu_q)
     tq, hq, d = q.shape
     g = k_conv.shape[1]
     s = hq // g

@@ -1,0 +1,145 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py
+times: integer outputs (routes, indices, page tables, gathered bytes) are
+checked in full; attention outputs on seeded samples of rows that the oracle
+computes one by one.  Oracle inputs are the seeded host inputs and the seeded
+device-drawn cache / page contents (inputs, not results of the CUDA path)."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+from oracle import recache_oracle as orc
+from paper_2608_19662_b200 import workloads as wl
+
+from pipeline import f64, gpu_compact, gpu_encode, gpu_prefill, make_ctx, oracle_cache_only, sample_rows
+from test_gpu_parity import assert_rotated_close
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-2
+HALF_ULP = 2.0 ** -8     # outputs are bf16 here: half a unit in the last place of the reference on top
+
+
+def _close(got, ref):
+    return (np.abs(got - ref) <= TOL + HALF_ULP * np.abs(ref)).all()
+
+
+def test_bench_step_full_size():
+    import bench
+    w = bench.Workload("full")
+    run = bench.Runner(w, 0)
+    run.step()
+    torch.cuda.synchronize()
+    assert run.rc.poll_status() == 0
+    sh, pool, req, dc = w.shape, w.pool, w.req, w.dc
+    assert len(pool.lens) == 64 and pool.lens.min() >= 1000 and req.total_q == 2048 and dc.batch == 64
+    rng = np.random.default_rng(123)
+
+    # ---- encode: cache in full, outputs on sampled rows (tile-boundary tokens included) ----
+    kc_ref, vc_ref = oracle_cache_only(pool)
+    assert np.array_equal(f64(run.v_cache), vc_ref)
+    assert_rotated_close(sh, run.k_cache, kc_ref)
+    extra = [int(pool.cu_seqlens[i]) + t for i in (0, 17, 63) for t in (31, 32, 63, 64, 127, 128, 129, 999)]
+    rows = sample_rows(rng, pool.cu_seqlens, sh.n_q_heads, 260, extra_tokens=extra)
+    f32 = lambda t: t.float().numpy()            # bf16 values are exact in fp32; the oracle widens what it samples
+    ref = orc.encode_rows(f32(pool.q), f32(pool.k), f32(pool.v), pool.cu_seqlens, sh.rope_theta, rows, storage="bf16")
+    o = run.o_enc.cpu()
+    got = np.stack([f64(o[t, h]) for t, h in rows])
+    assert _close(got, ref)
+
+    # ---- packed compaction: exact ----
+    rt = orc.compact_routes(pool.keep, req.res_off, req.res_slot, req.res_len, req.vis)
+    cu = orc.route_prefix(rt)
+    assert np.array_equal(run.route_cu.cpu().numpy(), cu)
+    flat = np.concatenate([r for per in rt for r in per])
+    assert np.array_equal(run.route_idx.cpu().numpy()[:cu[-1]], flat)
+    g_of = np.concatenate([np.full(len(r), kg) for per in rt for kg, r in enumerate(per)])
+    gi, ri = torch.from_numpy(g_of).cuda().long(), torch.from_numpy(flat).cuda().long()
+    assert torch.equal(run.k_route.view(torch.int16)[:cu[-1]], run.k_cache.view(torch.int16)[gi, ri])
+    assert torch.equal(run.v_route.view(torch.int16)[:cu[-1]], run.v_cache.view(torch.int16)[gi, ri])
+    assert 0.05 < cu[-1] / (sh.n_kv_heads * pool.total_tokens) < 0.11          # ~8 % of the KV is retained
+
+    # ---- prefill: sampled rows ----
+    prow = sample_rows(rng, req.cu_q, sh.n_q_heads, 160, extra_tokens=[31, 32, 63, 64, 1023, 1024])
+    pref = orc.prefill_rows(f32(req.q), f32(req.k_conv), f32(req.v_conv), req.cu_q, req.q_pos0, rt, kc_ref, vc_ref,
+                            sh.rope_theta, prow, storage="bf16")
+    op = run.o_pre.cpu()
+    assert _close(np.stack([f64(op[t, h]) for t, h in prow]), pref)
+
+    # ---- paged compaction for the decode batch: exact ----
+    rows4 = orc.compact_routes(dc.keep, dc.res_off, dc.dst_slot, dc.lens, dc.vis)
+    cu4 = orc.route_prefix(rows4)
+    assert np.array_equal(run.d_route_cu.cpu().numpy(), cu4)
+    assert np.array_equal(run.d_route_len.cpu().numpy(), np.diff(cu4))
+    flat4 = np.concatenate([r for per in rows4 for r in per])
+    assert np.array_equal(run.d_route_idx.cpu().numpy()[:cu4[-1]], flat4)
+    table_ref, used = orc.page_layout(rows4, dc.free_pages, wl.PAGE_TOKENS, dc.max_res_pages)
+    assert used == len(dc.free_pages)
+    assert np.array_equal(run.d_page_table.cpu().numpy(), table_ref)
+
+    # ---- decode: sampled (sequence, group) items from the seeded cache / history contents ----
+    g, d, pt, s = sh.n_kv_heads, sh.head_dim, wl.PAGE_TOKENS, sh.group_size
+    kc4, vc4 = run.d_k_cache.cpu(), run.d_v_cache.cpu()            # seeded inputs drawn on the device
+    kp_in = wl.seeded_normal(79, (dc.n_pages, pt, d), sh.torch_dtype, device="cuda").cpu()   # history contents, as drawn
+    vp_in = wl.seeded_normal(80, (dc.n_pages, pt, d), sh.torch_dtype, device="cuda").cpu()
+    od = run.o_dec.cpu()
+    items = sorted(set([0, dc.batch * g - 1] + [int(v) for v in rng.integers(0, dc.batch * g, 22)]))
+    flat_rows = [r for per in rows4 for r in per]
+    for it in items:
+        b, kg = divmod(it, g)
+        r = flat_rows[it]
+        n_rp = (len(r) + pt - 1) // pt
+        hp = dc.hist_page_table[it]
+        # a private little page pool for this item: its resource pages, then its history pages
+        kpool = np.zeros((n_rp + len(hp), pt, d)); vpool = np.zeros_like(kpool)
+        ridx, hidx = torch.from_numpy(r).long(), torch.from_numpy(hp).long()
+        kpool[:n_rp].reshape(-1, d)[:len(r)] = f64(kc4[kg][ridx]); vpool[:n_rp].reshape(-1, d)[:len(r)] = f64(vc4[kg][ridx])
+        kpool[n_rp:] = f64(kp_in[hidx]); vpool[n_rp:] = f64(vp_in[hidx])
+        res_t = np.arange(n_rp, dtype=np.int32)[None, :]
+        hist_t = (n_rp + np.arange(len(hp), dtype=np.int32))[None, :]
+        hl = np.array([dc.hist_len[it]], np.int32)
+        qp = np.array([dc.q_pos[b]], np.int32)
+        orc.append_decode_kv(kpool, vpool, hist_t, hl, f64(w.dec_k_new[b:b + 1, kg:kg + 1]),
+                             f64(w.dec_v_new[b:b + 1, kg:kg + 1]), qp, sh.rope_theta, pt, storage="bf16")
+        ref_o = orc.attend_decode(f64(w.dec_q[b:b + 1, kg * s:(kg + 1) * s]), qp, kpool, vpool, res_t,
+                                  np.array([len(r)], np.int32), hist_t, hl, sh.rope_theta, pt, storage="bf16")
+        assert _close(f64(od[b, kg * s:(kg + 1) * s]), ref_o[0])
+
+
+def test_composition_reuse_full_size_layer():
+    """One layer of the composition-reuse workload at full size: a pool of 64
+    resources U[150,1200] encoded once, 16 requests of 4-12 pool resources in
+    random order with 256-1024 query tokens; sampled rows against the oracle and
+    exact compaction.  (The 36 layers differ only in their seeds and routes.)"""
+    layer = 7
+    pool = wl.config3_pool(layer=layer)
+    sh = pool.shape
+    req = wl.config3_requests(pool, layer=layer)
+    assert len(pool.lens) == 64 and req.n_requests == 16 and 256 <= np.diff(req.cu_q).min()
+    rc = make_ctx(sh, max_pos=16384)
+    o, kc, vc = gpu_encode(rc, pool, out_dtype=torch.bfloat16)
+    kc_ref, vc_ref = oracle_cache_only(pool)
+    assert_rotated_close(sh, kc, kc_ref)
+    rng = np.random.default_rng(layer)
+    rows = sample_rows(rng, pool.cu_seqlens, sh.n_q_heads, 200)
+    f32 = lambda t: t.float().numpy()
+    ref = orc.encode_rows(f32(pool.q), f32(pool.k), f32(pool.v), pool.cu_seqlens, sh.rope_theta, rows, storage="bf16")
+    oc = o.cpu()
+    assert _close(np.stack([f64(oc[t, h]) for t, h in rows]), ref)
+    rt = orc.compact_routes(pool.keep, req.res_off, req.res_slot, req.res_len, req.vis)
+    out = gpu_compact(rc, pool, req, kc, vc)
+    cu = orc.route_prefix(rt)
+    assert np.array_equal(out["route_cu"].cpu().numpy(), cu)
+    assert np.array_equal(out["route_idx"].cpu().numpy()[:cu[-1]], np.concatenate([r for per in rt for r in per]))
+    p, _, _ = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"], out_dtype=torch.bfloat16)
+    prow = sample_rows(rng, req.cu_q, sh.n_q_heads, 200)
+    pref = orc.prefill_rows(f32(req.q), f32(req.k_conv), f32(req.v_conv), req.cu_q, req.q_pos0, rt, kc_ref, vc_ref,
+                            sh.rope_theta, prow, storage="bf16")
+    pc = p.cpu()
+    assert _close(np.stack([f64(pc[t, h]) for t, h in prow]), pref)
+    assert rc.poll_status() == 0
