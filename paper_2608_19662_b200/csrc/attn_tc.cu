@@ -189,6 +189,22 @@ constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3
 constexpr uint32_t IDESC_QK = IDESC_BASE;               // A, B K-major
 constexpr uint32_t IDESC_PV = IDESC_BASE | (1u << 16);  // B (= V) MN-major
 
+// Packed fp32 pairs (one instruction, two lanes of the FMA pipe).
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
+  asm("{\n\t.reg .b64 ra, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\tadd.rn.f32x2 rd, rd, ra;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&p);
@@ -533,7 +549,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       }
       uint8_t* qb = sm_gen + SM_Q + x * TILE_BYTES + row * 128;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int cc = 0; cc < 8; ++cc) {
+        // threads of a warp read 8 different cos/sin rows 256 bytes apart: start each row at another chunk
+        const int c = (cc + row / s) & 7;
         const int off = ((c ^ (row & 7)) << 4);
         const uint4 ulo = *reinterpret_cast<uint4*>(qb + off), uhi = *reinterpret_cast<uint4*>(qb + BOX_BYTES + off);
         const float4 c0 = cp[2 * c], c1 = cp[2 * c + 1], s0 = sp[2 * c], s1 = sp[2 * c + 1];
@@ -581,10 +599,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           }
           float mx4[4] = {__uint_as_float(sr[0]), __uint_as_float(sr[1]), __uint_as_float(sr[2]), __uint_as_float(sr[3])};
 #pragma unroll
-          for (int c = 4; c < 128; c += 4) {
+          for (int c = 4; c < 124; c += 8) {     // three-input max: 4 chains, 2 new values per step
 #pragma unroll
-            for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sr[c + u]));
+            for (int u = 0; u < 4; ++u) mx4[u] = fmax3(mx4[u], __uint_as_float(sr[c + 2 * u]), __uint_as_float(sr[c + 2 * u + 1]));
           }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mx4[u] = fmaxf(mx4[u], __uint_as_float(sr[124 + u]));
           const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
           const float m_new = fmaxf(m_ref, mx);
           bool need = false;
@@ -611,11 +631,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
           for (int c = 0; c < 64; c += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sr[2 * c]), c2, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(sr[2 * c + 1]), c2, neg_m));
-            const float p2 = ex2(fmaf(__uint_as_float(sr[2 * c + 2]), c2, neg_m));
-            const float p3 = ex2(fmaf(__uint_as_float(sr[2 * c + 3]), c2, neg_m));
-            acc[0] += p0; acc[1] += p1; acc[2] += p2; acc[3] += p3;
+            float x0, x1, x2, x3;
+            fma2(x0, x1, __uint_as_float(sr[2 * c]), __uint_as_float(sr[2 * c + 1]), c2, neg_m);
+            fma2(x2, x3, __uint_as_float(sr[2 * c + 2]), __uint_as_float(sr[2 * c + 3]), c2, neg_m);
+            const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+            add2(acc[0], acc[1], p0, p1);
+            add2(acc[2], acc[3], p2, p3);
             pr[c] = pack2(p0, p1);
             pr[c + 1] = pack2(p2, p3);
             if (c == 30) TMEM_ST32(t_s + 0, pr, 0);        // first half of P goes out while the second is computed
