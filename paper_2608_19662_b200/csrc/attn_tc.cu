@@ -39,7 +39,7 @@ constexpr int NSTAGE = 2;
 constexpr int BOX_BYTES = 16384;   // [128 rows][64 bf16], 128-byte swizzle
 constexpr int TILE_BYTES = 32768;  // two boxes: head_dim halves
 constexpr int NTHREADS = 384;
-constexpr int REGS_SOFTMAX = 216, REGS_AUX = 72;   // 256*224 + 128*56 = 384*168
+constexpr int REGS_SOFTMAX = 224, REGS_AUX = 56;   // 256*224 + 128*56 = 384*168
 
 constexpr int SM_Q = 0;                              // 2 query tiles
 constexpr int SM_K = SM_Q + 2 * TILE_BYTES;          // NSTAGE key tiles
