@@ -6,9 +6,10 @@
 //              every visible resource inside its route, the page prefix and
 //              the page table (one CTA; a few thousand integers)
 //   3. gather: one CTA per (listed resource, group) that the route table marks
-//              visible: stable stream compaction of the keep mask (block scan),
-//              the row indices, and 16-byte-vectorised copies of the kept key
-//              and value rows into the packed or paged destination.
+//              visible: stable stream compaction of the keep mask (one block
+//              scan per 2048 tokens), the row indices, and 16-byte-vectorised
+//              copies of the kept key and value rows into the packed or paged
+//              destination, eight pieces in flight per thread.
 // Order inside a route = request order, then ascending token (stable), so the
 // indices are unique and can be compared bit for bit.
 #include "common.cuh"
@@ -135,6 +136,13 @@ __global__ void __launch_bounds__(1024) compact_plan_kernel(
   }
 }
 
+constexpr int TOK_PER_THREAD = 8;
+constexpr int SUPER = TPB * TOK_PER_THREAD;   // tokens scanned per pass (2048)
+
+// One CTA per (listed resource, group) that the route table marks visible.
+// Pass = up to 2048 tokens: every thread reads 8 mask bytes, one block scan ranks
+// the kept tokens, their (source row, destination row) pairs go to shared memory,
+// and then all threads stream the rows with eight 16-byte pieces in flight each.
 __global__ void __launch_bounds__(TPB) compact_gather_kernel(
     const uint8_t* __restrict__ k_cache, const uint8_t* __restrict__ v_cache, int64_t pool_tokens,
     const uint8_t* __restrict__ keep, const int32_t* __restrict__ res_off,
@@ -145,8 +153,8 @@ __global__ void __launch_bounds__(TPB) compact_gather_kernel(
     uint8_t* __restrict__ k_out, uint8_t* __restrict__ v_out, const int32_t* __restrict__ free_pages,
     int64_t n_free_pages, int64_t n_pool_pages, int row_bytes) {
   __shared__ int ws[TPB / 32 + 1];
-  __shared__ int64_t src_row[TPB];   // cache row of the chunk's n-th kept token
-  __shared__ int64_t dst_row[TPB];   // destination row (packed row, or page*page_tokens+slot); -1 = skip
+  __shared__ int32_t src_tok[SUPER];   // token offset (inside the resource) of the pass's n-th kept token
+  __shared__ int32_t dst_row[SUPER];   // destination row (packed row, or page * page_tokens + slot); -1 = skip
   const int r = blockIdx.x, g = blockIdx.y;
   if (!vis[(int64_t)g * total_listed + r]) return;
   const int64_t s0 = res_slot[r];
@@ -158,43 +166,68 @@ __global__ void __launch_bounds__(TPB) compact_gather_kernel(
   const int64_t route_base = route_cu[route];
   const int64_t page_base = page_cu[route];
   const int segs = row_bytes / 16;
-  const uint8_t* kc = k_cache + (int64_t)g * pool_tokens * row_bytes;
-  const uint8_t* vc = v_cache + (int64_t)g * pool_tokens * row_bytes;
+  const uint8_t* kc = k_cache + ((int64_t)g * pool_tokens + s0) * row_bytes;
+  const uint8_t* vc = v_cache + ((int64_t)g * pool_tokens + s0) * row_bytes;
 
   int run = 0;
-  for (int j0 = 0; j0 < n; j0 += TPB) {
-    const int j = j0 + threadIdx.x;
-    const int flag = (j < n) && keep[s0 + j] != 0;
+  for (int j0 = 0; j0 < n; j0 += SUPER) {
+    const int jt = j0 + threadIdx.x * TOK_PER_THREAD;
+    uint32_t flags = 0;
+#pragma unroll
+    for (int u = 0; u < TOK_PER_THREAD; ++u)
+      if (jt + u < n && keep[s0 + jt + u] != 0) flags |= 1u << u;
     int tot;
-    const int ex = block_excl_scan(flag, ws, &tot);
-    if (flag) {
-      const int rank = in_route + run + ex;              // row inside the route
-      const int64_t packed = route_base + rank;
-      if (packed < row_capacity) route_idx[packed] = (int32_t)(s0 + j);
-      int64_t dst = -1;
-      if (mode == RECACHE_PACKED) {
-        if (packed < row_capacity) dst = packed;
-      } else {
-        const int64_t fi = page_base + rank / page_tokens;
-        if (fi < n_free_pages) {
-          const int pg = free_pages[fi];
-          if (pg >= 0 && pg < n_pool_pages) dst = (int64_t)pg * page_tokens + rank % page_tokens;
+    int rank = in_route + run + block_excl_scan(__popc(flags), ws, &tot);   // row inside the route
+    const int list0 = rank - in_route - run;
+    int k = 0;
+#pragma unroll
+    for (int u = 0; u < TOK_PER_THREAD; ++u) {
+      if (flags & (1u << u)) {
+        const int64_t packed = route_base + rank;
+        if (packed < row_capacity && blockIdx.z == 0) route_idx[packed] = (int32_t)(s0 + jt + u);
+        int64_t dst = -1;
+        if (mode == RECACHE_PACKED) {
+          if (packed < row_capacity) dst = packed;
+        } else {
+          const int64_t fi = page_base + rank / page_tokens;
+          if (fi < n_free_pages) {
+            const int pg = free_pages[fi];
+            if (pg >= 0 && pg < n_pool_pages) dst = (int64_t)pg * page_tokens + rank % page_tokens;
+          }
         }
+        src_tok[list0 + k] = jt + u;
+        dst_row[list0 + k] = (int32_t)dst;
+        ++k; ++rank;
       }
-      src_row[ex] = s0 + j;
-      dst_row[ex] = dst;
     }
     __syncthreads();
-    // cooperative 16-byte copies: consecutive threads move consecutive pieces of a row
-    for (int e = threadIdx.x; e < tot * segs; e += TPB) {
-      const int rr = e / segs, sg = e - rr * segs;
-      const int64_t d = dst_row[rr];
-      if (d < 0) continue;
-      const int64_t so = src_row[rr] * row_bytes + sg * 16, dof = d * row_bytes + sg * 16;
-      const uint4 kx = *reinterpret_cast<const uint4*>(kc + so);
-      const uint4 vx = *reinterpret_cast<const uint4*>(vc + so);
-      *reinterpret_cast<uint4*>(k_out + dof) = kx;
-      *reinterpret_cast<uint4*>(v_out + dof) = vx;
+    // with few (resource, group) pairs the copy is shared by gridDim.z CTAs that all ran the (cheap) scan
+    const int n_piece = tot * segs;
+    for (int e0 = threadIdx.x + blockIdx.z * TPB * 4; e0 < n_piece; e0 += TPB * 4 * gridDim.z) {
+      uint4 kx[4], vx[4];
+      int64_t dof[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + u * TPB;
+        dof[u] = -1;
+        if (e < n_piece) {
+          const int rr = e / segs, sg = e - rr * segs;
+          const int d = dst_row[rr];
+          if (d >= 0) {
+            const int64_t so = (int64_t)src_tok[rr] * row_bytes + sg * 16;
+            dof[u] = (int64_t)d * row_bytes + sg * 16;
+            kx[u] = *reinterpret_cast<const uint4*>(kc + so);
+            vx[u] = *reinterpret_cast<const uint4*>(vc + so);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (dof[u] >= 0) {
+          *reinterpret_cast<uint4*>(k_out + dof[u]) = kx[u];
+          *reinterpret_cast<uint4*>(v_out + dof[u]) = vx[u];
+        }
+      }
     }
     run += tot;
     __syncthreads();
@@ -240,7 +273,9 @@ cudaError_t rc_launch_compact(const recache_ctx* ctx, const CompactArgs& a, cuda
                                             a.free_pages, a.n_free_pages, a.n_pool_pages, ctx->status);
   }
   if (a.total_listed > 0) {
-    dim3 grid((unsigned)a.total_listed, (unsigned)G);
+    const int64_t pairs = (int64_t)a.total_listed * G;
+    const unsigned z = (unsigned)(pairs >= 2048 ? 1 : (2048 + pairs - 1) / pairs > 8 ? 8 : (2048 + pairs - 1) / pairs);
+    dim3 grid((unsigned)a.total_listed, (unsigned)G, z);
     RcLaunchScope scope(ctx, RC_K_COMPACT_GATHER, st);
     compact_gather_kernel<<<grid, TPB, 0, st>>>(
         (const uint8_t*)a.k_cache, (const uint8_t*)a.v_cache, a.pool_tokens, a.keep, a.res_off, a.res_slot,
