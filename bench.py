@@ -206,7 +206,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.p = None
@@ -239,17 +239,19 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------- oracle sample --
-def oracle_sample(w: Workload, budget: str = "default"):
+def oracle_sample(w: Workload, frac: float = 1.0):
     """Times the fp64 oracle, as it stands, on a bounded sample of the same
     workload: whole resources for a few heads (encode), a block of query tokens
-    (prefill) and a few decode items.  Returns (flops, seconds, description)."""
+    (prefill) and a few decode items.  frac = 1 is about 10-20 s of CPU work;
+    the reference arm shrinks it so that all its steps fit in a few minutes.
+    Returns (flops, seconds, description)."""
     from oracle import recache_oracle as orc
     sh = w.shape
     p, r, dc = w.pool, w.req, w.dc
     d, s = sh.head_dim, sh.group_size
     f64 = lambda t: t.to(torch.float64).numpy()
-    n_res = min(12, len(p.lens))
-    ng = min(2, sh.n_kv_heads)
+    ng = min(sh.n_kv_heads, 4 if frac >= 0.5 else 2 if frac >= 0.12 else 1)
+    n_res = min(len(p.lens), max(1, int(round(96 * frac / ng))))
     t_end = int(p.cu_seqlens[n_res])
     t0 = time.perf_counter()
     # encode: first n_res resources, query heads of the first ng KV groups
@@ -262,12 +264,12 @@ def oracle_sample(w: Workload, budget: str = "default"):
     kc = np.zeros((1, p.pool_tokens, d)); vc = np.zeros_like(kc)
     rng = np.random.default_rng(0)
     kc[0, rows[0][0]] = rng.standard_normal((len(rows[0][0]), d)); vc[0, rows[0][0]] = 1.0
-    tq = min(512, r.total_q)
+    tq = min(max(64, int(1024 * frac)), r.total_q)
     orc.attend_prefill(f64(r.q[:tq, :s]), f64(r.k_conv[:tq, :1]), f64(r.v_conv[:tq, :1]), [0, tq], r.q_pos0, rows,
                        kc, vc, sh.rope_theta, storage=sh.dtype)
     flops += 4 * d * s * (tq * len(rows[0][0]) + tq * (tq + 1) // 2)
     # decode: 8 items over synthetic pages of the workload's lengths
-    n_it = 32
+    n_it = max(4, int(64 * frac))
     hist = int(dc.hist_len[0]); res = 720 if hist >= 2048 else 200
     pt = wl.PAGE_TOKENS
     n_pg = n_it * ((hist + pt - 1) // pt + (res + pt - 1) // pt)
@@ -289,11 +291,13 @@ def run_reference(args):
     if rank != 0:
         return
     w = Workload(args.case)
+    # a full sample is ~10 s of CPU work here: shrink it so that steps + warm-up take about 2.5 minutes
+    frac = min(1.0, max(0.02, 150.0 / (10.0 * max(1, args.steps + args.warmup))))
     for _ in range(args.warmup):
-        oracle_sample(w)
+        oracle_sample(w, frac)
     t0 = time.perf_counter(); fl = 0
     for _ in range(args.steps):
-        f, _, what = oracle_sample(w)
+        f, _, what = oracle_sample(w, frac)
         fl += f
     sec = time.perf_counter() - t0
     val = fl / sec / 1e12
@@ -328,7 +332,7 @@ def job_value(world: int, flops_per_rank: float, ms_step: float) -> float:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default="full", choices=["full", "medium", "small"],
