@@ -154,6 +154,29 @@ RECACHE_API recache_status recache_encode_resources(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
+ * Encoding variants of the paper's ablation (section "Cache Reuse"): resources
+ * "pre-encoded with a shared prefix", and the "Block" configuration that drops
+ * cross-resource attention but keeps the original positional indices.
+ * Same as recache_encode_resources, plus
+ *   k_prefix / v_prefix [G][prefix_len][d]: rotated keys and values of a shared
+ *       prefix, as a cache holds them (e.g. written by an earlier encode call);
+ *       every resource token also attends to all of them ("attend only to the
+ *       shared prefix and their local resource tokens").  NULL / 0: no prefix.
+ *   pos_offset [N] (device, may be NULL = all 0): position of each resource's
+ *       first token.  One common value P = the resource-local layout behind a
+ *       prefix of P tokens (still composition-independent); global offsets = the
+ *       "Block" variant.  Positions pos_offset[i] + D_i must stay below max_pos.
+ * The cache receives keys rotated at those positions.
+ */
+RECACHE_API recache_status recache_encode_resources_prefixed(recache_ctx* ctx,
+    const void* q, const void* k, const void* v,
+    const int32_t* cu_seqlens, int32_t n_resources, int32_t total_tokens, int32_t max_len,
+    const int32_t* dst_slot, void* k_cache, void* v_cache, int64_t pool_tokens,
+    const void* k_prefix, const void* v_prefix, int32_t prefix_len, const int32_t* pos_offset,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
  * Route / keep-mask compaction = request-local KV materialisation (paper:
  * "Structural Pruning", "Semantic Pruning", and the TTFT definition).
  * Request b lists resources res_off[b] .. res_off[b+1]-1 (entries of res_slot /

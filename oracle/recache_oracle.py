@@ -89,10 +89,16 @@ def _softmax_rows(s: np.ndarray) -> np.ndarray:
 
 # ----------------------------------------------------------------- encode --
 def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] = None,
-                     pos_offset: Optional[Sequence[int]] = None):
+                     pos_offset: Optional[Sequence[int]] = None, prefix_k=None, prefix_v=None):
     """Resource-wise encoding.  q: [T,Hq,d]; k, v: [T,G,d] (pre-RoPE), resource
-    i = rows cu_seqlens[i]..cu_seqlens[i+1]-1 at local positions 0..D_i-1
-    (+ pos_offset[i], used only to pin shift invariance).
+    i = rows cu_seqlens[i]..cu_seqlens[i+1]-1 at positions pos_offset[i] + 0..D_i-1
+    (pos_offset = None: resource-local positions from 0; one common offset P: the
+    layout after a shared prefix of P tokens; global offsets: the "Block"
+    variant, which drops cross-resource attention but keeps original positions).
+    prefix_k / prefix_v [G][P][d]: rotated keys / values of a shared prefix as a
+    cache holds them; every resource token sees all of them besides its own
+    resource's tokens j' <= j ("attend only to the shared prefix and their local
+    resource tokens").
     Returns (o [T,Hq,d], k_hat [T,G,d] in storage precision, v [T,G,d])."""
     q = np.asarray(q, F64); k = np.asarray(k, F64); v = np.asarray(v, F64)
     t, hq, d = q.shape
@@ -114,7 +120,12 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
             kg = h // s
             sc = qh[:, h, :] @ kh[:, kg, :].T / math.sqrt(d)
             sc = np.where(causal, sc, -np.inf)
-            o[a:b, h, :] = _softmax_rows(sc) @ v[a:b, kg, :]
+            vals = v[a:b, kg, :]
+            if prefix_k is not None and np.asarray(prefix_k).shape[1] > 0:
+                pk, pv = np.asarray(prefix_k[kg], F64), np.asarray(prefix_v[kg], F64)
+                sc = np.concatenate([qh[:, h, :] @ pk.T / math.sqrt(d), sc], axis=1)
+                vals = np.concatenate([pv, vals], axis=0)
+            o[a:b, h, :] = _softmax_rows(sc) @ vals
     return o, k_hat, v.copy()
 
 

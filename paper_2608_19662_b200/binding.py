@@ -45,6 +45,8 @@ SIGNATURES = {
     "recache_decode_workspace_bytes": (_I64, [_P, _I32, _I32, _I32]),
     "recache_encode_resources": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _I32,
                                            _P, _I64, _P]),
+    "recache_encode_resources_prefixed": (C.c_int, [_P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
+                                                    _I32, _P, _P, _I32, _P, _I64, _P]),
     "recache_compact_routes": (C.c_int, [_P, _P, _P, _I64, _P, _P, _P, _P, _I32, _I32, _P, _I32, _P, _P, _P,
                                          _I64, _P, _P, _P, _I32, _P, _I64, _I64, _P, _I64, _P]),
     "recache_attend_prefill": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
@@ -177,6 +179,23 @@ class ReCache:
                                                int(max_len), _ptr(dst_slot), _ptr(k_cache), _ptr(v_cache),
                                                k_cache.shape[1], _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_encode_resources")
+        return out
+
+    def encode_resources_prefixed(self, q, k, v, cu_seqlens, max_len, dst_slot, k_cache, v_cache, k_prefix=None,
+                                  v_prefix=None, pos_offset=None, out=None, out_dtype=None, workspace=None):
+        """recache_encode_resources_prefixed: encode behind a shared prefix [G,P,d] and / or with a first
+        position per resource (pos_offset [N]).  Returns o [T,Hq,d]."""
+        n_res = cu_seqlens.numel() - 1
+        total = q.shape[0]
+        od, oc = self._out_code(out_dtype)
+        if out is None:
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        ws = workspace if workspace is not None else self.workspace(self.encode_workspace_bytes(n_res, total, max_len))
+        st = self.lib.recache_encode_resources_prefixed(
+            self.h, _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), n_res, total, int(max_len), _ptr(dst_slot),
+            _ptr(k_cache), _ptr(v_cache), k_cache.shape[1], _ptr(k_prefix), _ptr(v_prefix),
+            0 if k_prefix is None else k_prefix.shape[1], _ptr(pos_offset), _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
+        self._check(st, "recache_encode_resources_prefixed")
         return out
 
     def compact_routes(self, k_cache, v_cache, keep, res_off, res_slot, res_len, vis, mode, route_cu, route_idx,

@@ -145,12 +145,16 @@ int64_t recache_decode_workspace_bytes(const recache_ctx* ctx, int32_t batch, in
   return rc_decode_workspace_bytes(ctx, batch, max_res_pages, max_hist_pages);
 }
 
-recache_status recache_encode_resources(recache_ctx* ctx, const void* q, const void* k, const void* v,
-                                        const int32_t* cu_seqlens, int32_t n_resources, int32_t total_tokens,
-                                        int32_t max_len, const int32_t* dst_slot, void* k_cache, void* v_cache,
-                                        int64_t pool_tokens, void* out_o, int32_t out_dtype, void* workspace,
-                                        int64_t workspace_bytes, void* stream) {
+static recache_status encode_impl(recache_ctx* ctx, const void* q, const void* k, const void* v,
+                                  const int32_t* cu_seqlens, int32_t n_resources, int32_t total_tokens,
+                                  int32_t max_len, const int32_t* dst_slot, void* k_cache, void* v_cache,
+                                  int64_t pool_tokens, const void* k_prefix, const void* v_prefix,
+                                  int32_t prefix_len, const int32_t* pos_offset, void* out_o, int32_t out_dtype,
+                                  void* workspace, int64_t workspace_bytes, void* stream) {
   if (!ctx) return RECACHE_EINVAL;
+  RC_REQUIRE(prefix_len >= 0, RECACHE_EINVAL, "encode: negative prefix_len");
+  RC_REQUIRE(prefix_len == 0 || (k_prefix && v_prefix && aligned16(k_prefix) && aligned16(v_prefix)), RECACHE_EINVAL,
+             "encode: prefix tensors missing or not 16-byte aligned");
   RC_REQUIRE(n_resources >= 0 && total_tokens >= 0 && max_len >= 0 && pool_tokens >= 0, RECACHE_EINVAL,
              "encode: negative size");
   RC_REQUIRE(out_dtype_ok(ctx, out_dtype), RECACHE_EINVAL, "encode: out_dtype must be f32 or the context dtype");
@@ -165,13 +169,34 @@ recache_status recache_encode_resources(recache_ctx* ctx, const void* q, const v
   cudaStream_t st = (cudaStream_t)stream;
   RC_CUDA(cudaSetDevice(ctx->device), "encode: set device");
 
-  RopeStoreArgs ra{k, v, k_cache, v_cache, cu_seqlens, n_resources, total_tokens, dst_slot, nullptr,
+  RopeStoreArgs ra{k, v, k_cache, v_cache, cu_seqlens, n_resources, total_tokens, dst_slot, pos_offset,
                    pool_tokens, 0};
   RC_CUDA(rc_launch_rope_store(ctx, ra, st), "encode: rope/store launch");
   EncodeArgs ea{q, out_o, out_dtype, cu_seqlens, n_resources, total_tokens, max_len, dst_slot,
-                k_cache, v_cache, pool_tokens, workspace, workspace_bytes};
+                k_cache, v_cache, pool_tokens, workspace, workspace_bytes, k_prefix, v_prefix, prefix_len, pos_offset};
   RC_CUDA(rc_launch_encode_attn(ctx, ea, st), "encode: attention launch");
   return RECACHE_OK;
+}
+
+recache_status recache_encode_resources(recache_ctx* ctx, const void* q, const void* k, const void* v,
+                                        const int32_t* cu_seqlens, int32_t n_resources, int32_t total_tokens,
+                                        int32_t max_len, const int32_t* dst_slot, void* k_cache, void* v_cache,
+                                        int64_t pool_tokens, void* out_o, int32_t out_dtype, void* workspace,
+                                        int64_t workspace_bytes, void* stream) {
+  return encode_impl(ctx, q, k, v, cu_seqlens, n_resources, total_tokens, max_len, dst_slot, k_cache, v_cache,
+                     pool_tokens, nullptr, nullptr, 0, nullptr, out_o, out_dtype, workspace, workspace_bytes, stream);
+}
+
+recache_status recache_encode_resources_prefixed(recache_ctx* ctx, const void* q, const void* k, const void* v,
+                                                 const int32_t* cu_seqlens, int32_t n_resources,
+                                                 int32_t total_tokens, int32_t max_len, const int32_t* dst_slot,
+                                                 void* k_cache, void* v_cache, int64_t pool_tokens,
+                                                 const void* k_prefix, const void* v_prefix, int32_t prefix_len,
+                                                 const int32_t* pos_offset, void* out_o, int32_t out_dtype,
+                                                 void* workspace, int64_t workspace_bytes, void* stream) {
+  return encode_impl(ctx, q, k, v, cu_seqlens, n_resources, total_tokens, max_len, dst_slot, k_cache, v_cache,
+                     pool_tokens, k_prefix, v_prefix, prefix_len, pos_offset, out_o, out_dtype, workspace,
+                     workspace_bytes, stream);
 }
 
 recache_status recache_compact_routes(recache_ctx* ctx, const void* k_cache, const void* v_cache,

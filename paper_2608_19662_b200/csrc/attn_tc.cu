@@ -65,6 +65,7 @@ struct TcParams {
   const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter
   const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu;
   int n_seq, G, Hq, s;
+  int prefix_len;   // > 0: every sequence sees rows g*prefix_len .. of the "route" tensors (shared prefix)
   int64_t self_rows;
   void* out;
   const float* cos_tab; const float* sin_tab; int max_pos;
@@ -277,6 +278,7 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
   it.pos0 = p.pos0 ? p.pos0[b] : 0;
   it.rA0 = 0; it.lenA = 0;
   if (p.route_cu) { it.rA0 = p.route_cu[b * p.G + it.g]; it.lenA = p.route_cu[b * p.G + it.g + 1] - it.rA0; }
+  else if (p.prefix_len > 0) { it.rA0 = it.g * p.prefix_len; it.lenA = p.prefix_len; }
   it.nA = (it.lenA + TILE_N - 1) / TILE_N;
   it.n_tiles = it.nA + (it.kv_end + TILE_N - 1) / TILE_N;
   const bool ok = it.L > 0 && it.tok0 < it.L && it.lenA >= 0 && it.rA0 >= 0 && it.base >= 0 &&
@@ -329,7 +331,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   }
   if (warp == 8 && lane == 0) {
     prefetch_tmap(&tm_q); prefetch_tmap(&tm_ks); prefetch_tmap(&tm_vs);
-    if (p.route_cu) { prefetch_tmap(&tm_kr); prefetch_tmap(&tm_vr); }
+    if (p.route_cu || p.prefix_len > 0) { prefetch_tmap(&tm_kr); prefetch_tmap(&tm_vr); }
   }
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sm + SM_MISC), "r"(512u) : "memory");
@@ -775,7 +777,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   if (!map_q(&tq, a.q, (uint64_t)a.total, Hq, s) || !map_rows(&tks, a.k_self, self_total) ||
       !map_rows(&tvs, a.v_self, self_total))
     return cudaErrorInvalidValue;
-  const bool has_route = a.route_cu != nullptr && a.route_rows > 0;
+  const bool has_route = (a.route_cu != nullptr || a.prefix_len > 0) && a.route_rows > 0;
   if (!map_rows(&tkr, has_route ? a.k_route : a.k_self, has_route ? (uint64_t)a.route_rows : self_total) ||
       !map_rows(&tvr, has_route ? a.v_route : a.v_self, has_route ? (uint64_t)a.route_rows : self_total))
     return cudaErrorInvalidValue;
@@ -788,6 +790,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   TcParams p;
   p.items = items; p.header = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
   p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.out = a.o;
+  p.prefix_len = a.route_cu ? 0 : a.prefix_len;
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)ctx->desc.head_dim));
   p.status = ctx->status;

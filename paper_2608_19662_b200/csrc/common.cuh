@@ -75,14 +75,15 @@ template <> __device__ __forceinline__ __nv_bfloat16 rc_from_float<__nv_bfloat16
 // All return the cudaError_t of the launch (cudaGetLastError).
 
 // Rotates keys at their positions and stores keys/values head-major.
-//  mode 0 (encode): token t of resource i -> position t - cu[i], row slot[i] + (t - cu[i])
+//  mode 0 (encode): token t of resource i -> position pos0[i] + t - cu[i] (pos0 may be null = 0),
+//                   row slot[i] + (t - cu[i])
 //  mode 1 (prefill): token t of request b -> position pos0[b] + (t - cu[b]), row t
 struct RopeStoreArgs {
   const void* k; const void* v;       // [total][G][d]
   void* k_dst; void* v_dst;           // [G][dst_rows][d]
   const int32_t* cu; int n_seq; int total;
   const int32_t* slot;                // mode 0
-  const int32_t* pos0;                // mode 1
+  const int32_t* pos0;                // mode 1; optional in mode 0
   int64_t dst_rows;
   int mode;
 };
@@ -98,6 +99,7 @@ struct AttnRowsArgs {
   const void* k_self; const void* v_self;  // [G][self_rows][d] rotated keys / values
   int64_t self_rows;
   const void* k_route; const void* v_route; const int32_t* route_cu;  // null for encode
+  int prefix_len;   // > 0 (with route_cu null): every sequence sees rows g*prefix_len .. +prefix_len of k_route/v_route
 };
 cudaError_t rc_launch_attn_rows(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t st);
 
@@ -134,6 +136,8 @@ struct EncodeArgs {
   const int32_t* cu; int n_res; int total; int max_len;
   const int32_t* slot; const void* k_cache; const void* v_cache; int64_t pool_tokens;
   void* workspace; int64_t workspace_bytes;
+  const void* k_prefix; const void* v_prefix; int prefix_len;   // shared prefix [G][prefix_len][d], or null / 0
+  const int32_t* pos_offset;                                      // first position of each resource, or null
 };
 struct PrefillArgs {
   const void* q; void* o; int out_dtype;
@@ -158,6 +162,7 @@ struct TcAttnArgs {
   const void* k_self; const void* v_self; int64_t self_rows;   // [G][self_rows][128]
   const void* k_route; const void* v_route; const int32_t* route_cu; int64_t route_rows;
   void* workspace;
+  int prefix_len;   // > 0 (route_cu null): all sequences see rows g*prefix_len .. of k_route/v_route ([G*prefix_len][128])
 };
 bool rc_tc_supported(const recache_ctx* ctx);
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);

@@ -17,23 +17,24 @@ int64_t rc_decode_workspace_bytes(const recache_ctx* ctx, int batch, int max_res
 
 cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, cudaStream_t st) {
   if (rc_tc_supported(ctx)) {
-    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, a.max_len, nullptr, a.slot, a.k_cache, a.v_cache,
-                 a.pool_tokens, nullptr, nullptr, nullptr, 0, a.workspace};
+    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, a.max_len, a.pos_offset, a.slot, a.k_cache, a.v_cache,
+                 a.pool_tokens, a.k_prefix, a.v_prefix, nullptr, (int64_t)ctx->desc.n_kv_heads * a.prefix_len,
+                 a.workspace, a.prefix_len};
     return rc_launch_attn_tc(ctx, t, st);
   }
-  AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, nullptr, a.slot, a.k_cache, a.v_cache,
-                 a.pool_tokens, nullptr, nullptr, nullptr};
+  AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, a.pos_offset, a.slot, a.k_cache, a.v_cache,
+                 a.pool_tokens, a.k_prefix, a.v_prefix, nullptr, a.prefix_len};
   return rc_launch_attn_rows(ctx, r, st);
 }
 
 cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a, cudaStream_t st) {
   if (rc_tc_supported(ctx)) {
     TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.max_q, a.pos0, nullptr, a.k_conv, a.v_conv,
-                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace};
+                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace, 0};
     return rc_launch_attn_tc(ctx, t, st);
   }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, nullptr, a.k_conv, a.v_conv,
-                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu};
+                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, 0};
   return rc_launch_attn_rows(ctx, r, st);
 }
 

@@ -1,8 +1,9 @@
 // Rotary embedding of keys + head-major store of keys and values.
 //
-// Encoding: token t of resource i has local position t - cu[i] and goes to cache
-// row slot[i] + that position (section "Resource-Wise Attention": positions
-// restart inside every resource).  Prefill: token t of request b has position
+// Encoding: token t of resource i has local position t - cu[i] (plus the
+// resource's position offset when one is given) and goes to cache row slot[i] +
+// local position (section "Resource-Wise Attention": positions restart inside
+// every resource).  Prefill: token t of request b has position
 // pos0[b] + (t - cu[b]) and goes to row t of the conversation KV.
 // Memory-bound: reads k, v once, writes both once; 16-byte accesses.
 #include "common.cuh"
@@ -64,9 +65,10 @@ __global__ void __launch_bounds__(256) rope_store_kernel(
 
   const int b = rc_find_segment(cu, n_seq, t);
   const int local = t - cu[b];
-  int pos; int64_t row;
-  if (mode == 0) { pos = local; row = (int64_t)slot[b] + local; }
-  else           { pos = pos0[b] + local; row = t; }
+  // position = the sequence's first position (0 when none is given) + index inside the sequence;
+  // row = the sequence's first cache row + that index (encode) or the token index itself (prefill)
+  const int pos = (pos0 ? pos0[b] : 0) + local;
+  const int64_t row = mode == 0 ? (int64_t)slot[b] + local : (int64_t)t;
   if (t >= cu[n_seq] || cu[b + 1] < cu[b]) { rc_set_status(status, RECACHE_DEV_BAD_SEQLENS); return; }
   if (row < 0 || row >= dst_rows) { rc_set_status(status, RECACHE_DEV_BAD_SLOT); return; }
   if (pos < 0 || pos >= max_pos) { rc_set_status(status, RECACHE_DEV_BAD_POS); return; }

@@ -429,3 +429,62 @@ def test_decode_equals_last_prefill_row_and_paged_equals_packed():
 def test_pair_counts():
     assert orc.useful_pairs_encode([1, 2, 3]) == 1 + 3 + 6
     assert orc.useful_pairs_prefill(4, 10) == 40 + 10
+
+
+# ------------------------------------------- shared prefix / global positions --
+def test_prefixed_encode_is_causal_attention_over_prefix_plus_resource():
+    """One resource behind a shared prefix of P tokens, positions P..P+L-1, equals
+    the resource rows of standard causal attention over [prefix ; resource]
+    (torch fp64 SDPA); without a prefix the extended call is the plain one."""
+    sh = wl.Shape(4, 2, 32, 1e4, "f32")
+    P, L = 11, 23
+    qp, kp, vp = wl.resource_tensors(5, 100, P, sh)
+    q, k, v = wl.resource_tensors(5, 0, L, sh)
+    pk = np.transpose(orc.rope(f64(kp), np.arange(P), sh.rope_theta), (1, 0, 2))       # [G][P][d], as a cache holds it
+    pv = np.transpose(f64(vp), (1, 0, 2))
+    o, k_hat, _ = orc.encode_resources(f64(q), f64(k), f64(v), [0, L], sh.rope_theta, pos_offset=[P],
+                                       prefix_k=pk, prefix_v=pv)
+    qa = torch.from_numpy(orc.rope(np.concatenate([f64(qp), f64(q)]), np.arange(P + L), sh.rope_theta))
+    ka = torch.from_numpy(orc.rope(np.concatenate([f64(kp), f64(k)]), np.arange(P + L), sh.rope_theta))
+    va = torch.from_numpy(np.concatenate([f64(vp), f64(v)]))
+    want = torch.nn.functional.scaled_dot_product_attention(
+        qa.permute(1, 0, 2)[None], ka.permute(1, 0, 2).repeat_interleave(2, 0)[None],
+        va.permute(1, 0, 2).repeat_interleave(2, 0)[None], is_causal=True)[0].permute(1, 0, 2).numpy()
+    assert np.allclose(o, want[P:], atol=1e-12)
+    assert np.allclose(k_hat, ka.numpy()[P:], atol=1e-13)
+    o0, _, _ = orc.encode_resources(f64(q), f64(k), f64(v), [0, L], sh.rope_theta)
+    o1, _, _ = orc.encode_resources(f64(q), f64(k), f64(v), [0, L], sh.rope_theta, pos_offset=[0],
+                                    prefix_k=np.zeros((2, 0, 32)), prefix_v=np.zeros((2, 0, 32)))
+    assert np.array_equal(o0, o1)
+
+
+def test_block_variant_no_cross_resource_attention_with_global_positions():
+    """Global position offsets ("Block"): still no pair across resources, so each
+    resource equals its own causal attention; with a prefix the offsets matter
+    (the relative position to the prefix changes) and the result is the masked
+    dense attention over [prefix ; all resources] with original positions."""
+    sh = wl.TINY_F32
+    lens = [9, 14, 6]
+    P = 5
+    parts = [wl.resource_tensors(13, r, n, sh) for r, n in enumerate(lens)]
+    qp, kp, vp = wl.resource_tensors(13, 50, P, sh)
+    q = np.concatenate([f64(p[0]) for p in parts]); k = np.concatenate([f64(p[1]) for p in parts])
+    v = np.concatenate([f64(p[2]) for p in parts])
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    offs = [P + int(cu[i]) for i in range(3)]                      # original positions after the prefix
+    pk = np.transpose(orc.rope(f64(kp), np.arange(P), sh.rope_theta), (1, 0, 2)); pv = np.transpose(f64(vp), (1, 0, 2))
+    o, _, _ = orc.encode_resources(q, k, v, cu, sh.rope_theta, pos_offset=offs, prefix_k=pk, prefix_v=pv)
+    t = int(cu[-1])
+    res_of = np.searchsorted(cu, np.arange(t), side="right") - 1
+    s = sh.group_size
+    for h in range(sh.n_q_heads):
+        g = h // s
+        qs = [brute_rope(list(q[n, h]), P + n, sh.rope_theta) for n in range(t)]
+        ks = [brute_rope(list(f64(kp)[n, g]), n, sh.rope_theta) for n in range(P)] + \
+             [brute_rope(list(k[n, g]), P + n, sh.rope_theta) for n in range(t)]
+        vs = [list(f64(vp)[n, g]) for n in range(P)] + [list(v[n, g]) for n in range(t)]
+        want = brute_attention(qs, ks, vs, lambda i, j: j < P or (res_of[j - P] == res_of[i] and j - P <= i))
+        assert np.allclose(o[:, h, :], np.array(want), atol=1e-12)
+    o_local, _, _ = orc.encode_resources(q, k, v, cu, sh.rope_theta, pos_offset=[P] * 3, prefix_k=pk, prefix_v=pv)
+    assert np.abs(o_local - o)[cu[1]:].max() > 1e-3                # offsets do matter once there is a prefix
+    assert np.allclose(o_local[:cu[1]], o[:cu[1]], atol=1e-12)     # ... except for the first resource (same offset)
