@@ -255,6 +255,24 @@ RECACHE_API recache_status recache_attend_decode(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
+ * Route table from contribution scores (paper: "Structural Pruning", the
+ * weights w_i = max(s_i,0) / sum_j max(s_j,0), TopK and Omega* = L* x G*;
+ * sparsity rho of "Structural Budget Analysis").  Host-only helper, all
+ * pointers are HOST memory.
+ *   s_layers [n_layers], s_groups [n_groups]: leave-one-in contributions (or
+ *       already-normalised weights); negative values count as 0
+ *   k_layers, k_groups: budgets K_L, K_G; ties go to the lower index
+ *   omega [n_layers][n_groups] (out): 1 where route (l, g) exposes the resources;
+ *       a layer's row, repeated over the request's resources, is that layer's
+ *       `vis` table for recache_compact_routes
+ *   cc_layers, cc_groups (out, optional): contribution coverage of the kept units
+ *   rho (out, optional): 1 - K_L K_G / (L G)
+ */
+RECACHE_API recache_status recache_build_routes(const double* s_layers, int32_t n_layers,
+    const double* s_groups, int32_t n_groups, int32_t k_layers, int32_t k_groups,
+    uint8_t* omega, double* cc_layers, double* cc_groups, double* rho);
+
+/*
  * Decode without any allocation.  (The paper has no counterpart: this is a
  * deployment variant of recache_attend_decode, same arguments minus the
  * workspace, same results.)

@@ -334,6 +334,25 @@ def attend_decode(q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page
     return o
 
 
+# ---------------------------------------------------------- route selection --
+def routes_from_contributions(s_layers, s_groups, k_layers: int, k_groups: int):
+    """Omega* = TopK_{K_L}(w_l) x TopK_{K_G}(w_g) with w_i = max(s_i, 0) / sum_j max(s_j, 0)
+    ("Structural Pruning"); ties go to the lower index.  Returns (omega [L][G],
+    kept layers, kept groups, CC of the kept layers, CC of the kept groups)."""
+    def top(s, k):
+        w = np.maximum(np.asarray(s, F64), 0.0)
+        w = w / w.sum() if w.sum() > 0 else w
+        order = sorted(range(len(w)), key=lambda i: (-w[i], i))[:k]
+        return order, float(sum(w[i] for i in order))
+    kl, ccl = top(s_layers, k_layers)
+    kg, ccg = top(s_groups, k_groups)
+    omega = np.zeros((len(s_layers), len(s_groups)), dtype=np.uint8)
+    for l in kl:
+        for g in kg:
+            omega[l, g] = 1
+    return omega, kl, kg, ccl, ccg
+
+
 # ------------------------------------------------------------ bookkeeping --
 def structural_sparsity(n_layers_kept: int, n_groups_kept: int, n_layers: int, n_groups: int) -> float:
     """rho(Omega) = 1 - |L*||G*| / (L G) for a product route set."""

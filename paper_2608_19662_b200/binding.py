@@ -53,6 +53,9 @@ SIGNATURES = {
                                          _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                         _P, _I32, _P, _I64, _P]),
+    "recache_build_routes": (C.c_int, [C.POINTER(C.c_double), _I32, C.POINTER(C.c_double), _I32, _I32, _I32,
+                                       C.POINTER(C.c_uint8), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                       C.POINTER(C.c_double)]),
     "recache_attend_decode_noalloc": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                                 _P, _I32, _P]),
 }
@@ -87,6 +90,22 @@ def _stream():
 
 class ReCacheError(RuntimeError):
     pass
+
+
+def build_routes(s_layers, s_groups, k_layers: int, k_groups: int):
+    """recache_build_routes (host only): returns (omega [L][G] uint8 numpy array, cc_layers, cc_groups, rho)."""
+    import numpy as np
+    lib = load_library()
+    sl = np.ascontiguousarray(s_layers, dtype=np.float64)
+    sg = np.ascontiguousarray(s_groups, dtype=np.float64)
+    omega = np.zeros((len(sl), len(sg)), dtype=np.uint8)
+    ccl, ccg, rho = C.c_double(), C.c_double(), C.c_double()
+    dp = lambda a: a.ctypes.data_as(C.POINTER(C.c_double))
+    st = lib.recache_build_routes(dp(sl), len(sl), dp(sg), len(sg), int(k_layers), int(k_groups),
+                                  omega.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(ccl), C.byref(ccg), C.byref(rho))
+    if st != 0:
+        raise ReCacheError(f"recache_build_routes: {STATUS_NAMES.get(st, st)}")
+    return omega, ccl.value, ccg.value, rho.value
 
 
 class ReCache:
