@@ -235,6 +235,28 @@ RECACHE_API recache_status recache_attend_prefill(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
+ * Routed prefill of a later turn (paper, problem setup: the input also holds the
+ * "preceding conversational history when available in multi-turn interactions").
+ * Same as recache_attend_prefill, with the conversation's rotated keys / values
+ * kept in a cache [G][cache_rows][d]: request b owns rows conv_slot[b] ..., of
+ * which the first hist_len[b] hold its earlier turns.  The new tokens attend to
+ * (i) the route's rows, (ii) ALL hist_len[b] earlier rows, (iii) new tokens
+ * t' <= t, in one softmax; their rotated keys / values are appended at rows
+ * conv_slot[b] + hist_len[b] + t.  q_pos0[b] is the position of the first NEW
+ * token.  With 64-aligned slots the cache doubles as the decode history pages
+ * (page id = (g * cache_rows + conv_slot[b]) / 64 + n).
+ */
+RECACHE_API recache_status recache_attend_prefill_history(recache_ctx* ctx,
+    const void* q, const void* k_conv, const void* v_conv,
+    const int32_t* cu_q, const int32_t* q_pos0,
+    int32_t n_requests, int32_t total_q, int32_t max_q,
+    const void* k_route, const void* v_route, const int32_t* route_cu, int64_t route_rows,
+    void* k_conv_cache, void* v_conv_cache, int64_t cache_rows,
+    const int32_t* conv_slot, const int32_t* hist_len,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
  * Routed decode (paper: the same mask "during decoding"; the Attn. latency of
  * the efficiency study).  One query token per sequence at position q_pos[b].
  * Item it = b * G + g reads res_len[it] rows through res_page_table[it][*] and

@@ -227,11 +227,13 @@ def gather_paged(cache, rows, page_table, n_pages: int, page_tokens: int, fill=0
 
 # ------------------------------------------------------- routed attention --
 def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta: float,
-                   storage: Optional[str] = None):
+                   storage: Optional[str] = None, hist_k=None, hist_v=None):
     """Conversation tokens of request b (positions q_pos0[b] + t) attend, in one
     softmax with scale 1/sqrt(d), to (i) every row of their route's compacted
     resource KV (cached rotated keys used as stored) and (ii) conversation
     tokens t' <= t.  A route without rows is the context-only mask.
+    hist_k[b] / hist_v[b] ([G][H_b][d], rotated keys as stored): earlier turns of
+    request b, all visible to every new token (multi-turn history).
     Returns (o [sum Tq,Hq,d], k_conv_hat [sum Tq,G,d] in storage precision)."""
     q = np.asarray(q, F64); k_conv = np.asarray(k_conv, F64); v_conv = np.asarray(v_conv, F64)
     tq, hq, d = q.shape
@@ -254,6 +256,9 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
             r = rows[b][kg]
             kr = np.asarray(k_cache[kg][r], F64).reshape(len(r), d)
             vr = np.asarray(v_cache[kg][r], F64).reshape(len(r), d)
+            if hist_k is not None and hist_k[b] is not None:     # earlier turns: more all-visible rows
+                kr = np.concatenate([kr, np.asarray(hist_k[b][kg], F64)], axis=0)
+                vr = np.concatenate([vr, np.asarray(hist_v[b][kg], F64)], axis=0)
             s_res = qh[:, h, :] @ kr.T / math.sqrt(d)
             s_conv = np.where(causal, qh[:, h, :] @ kh[:, kg, :].T / math.sqrt(d), -np.inf)
             p = _softmax_rows(np.concatenate([s_res, s_conv], axis=1))

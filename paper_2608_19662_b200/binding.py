@@ -51,6 +51,8 @@ SIGNATURES = {
                                          _I64, _P, _P, _P, _I32, _P, _I64, _I64, _P, _I64, _P]),
     "recache_attend_prefill": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
                                          _P, _I32, _P, _I64, _P]),
+    "recache_attend_prefill_history": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
+                                                 _I64, _P, _P, _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                         _P, _I32, _P, _I64, _P]),
     "recache_build_routes": (C.c_int, [C.POINTER(C.c_double), _I32, C.POINTER(C.c_double), _I32, _I32, _I32,
@@ -255,6 +257,23 @@ class ReCache:
                                              _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_attend_prefill")
         return out, k_conv_out, v_conv_out
+
+    def attend_prefill_history(self, q, k_conv, v_conv, cu_q, q_pos0, max_q, k_route, v_route, route_cu,
+                               k_conv_cache, v_conv_cache, conv_slot, hist_len, out=None, out_dtype=None, workspace=None):
+        """recache_attend_prefill_history: a later turn over caches [G,rows,d] that already hold hist_len[b]
+        rows per request from conv_slot[b]; appends the new rotated keys / values there.  Returns o."""
+        n_req = cu_q.numel() - 1
+        total_q = q.shape[0]
+        od, oc = self._out_code(out_dtype)
+        if out is None:
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        ws = workspace if workspace is not None else self.workspace(self.prefill_workspace_bytes(n_req, total_q, max_q))
+        st = self.lib.recache_attend_prefill_history(
+            self.h, _ptr(q), _ptr(k_conv), _ptr(v_conv), _ptr(cu_q), _ptr(q_pos0), n_req, total_q, int(max_q),
+            _ptr(k_route), _ptr(v_route), _ptr(route_cu), k_route.shape[0], _ptr(k_conv_cache), _ptr(v_conv_cache),
+            k_conv_cache.shape[1], _ptr(conv_slot), _ptr(hist_len), _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
+        self._check(st, "recache_attend_prefill_history")
+        return out
 
     def attend_decode(self, q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page_table, hist_len,
                       k_new=None, v_new=None, out=None, out_dtype=None, workspace=None):

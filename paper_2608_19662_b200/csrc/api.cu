@@ -231,14 +231,14 @@ recache_status recache_compact_routes(recache_ctx* ctx, const void* k_cache, con
   return RECACHE_OK;
 }
 
-recache_status recache_attend_prefill(recache_ctx* ctx, const void* q, const void* k_conv, const void* v_conv,
-                                      const int32_t* cu_q, const int32_t* q_pos0, int32_t n_requests,
-                                      int32_t total_q, int32_t max_q, const void* k_route, const void* v_route,
-                                      const int32_t* route_cu, int64_t route_rows, void* k_conv_out,
-                                      void* v_conv_out, void* out_o, int32_t out_dtype, void* workspace,
-                                      int64_t workspace_bytes, void* stream) {
+static recache_status prefill_impl(recache_ctx* ctx, const void* q, const void* k_conv, const void* v_conv,
+                                   const int32_t* cu_q, const int32_t* q_pos0, int32_t n_requests, int32_t total_q,
+                                   int32_t max_q, const void* k_route, const void* v_route, const int32_t* route_cu,
+                                   int64_t route_rows, void* k_conv_out, void* v_conv_out, int64_t conv_rows,
+                                   const int32_t* conv_slot, const int32_t* hist_len, void* out_o, int32_t out_dtype,
+                                   void* workspace, int64_t workspace_bytes, void* stream) {
   if (!ctx) return RECACHE_EINVAL;
-  RC_REQUIRE(n_requests >= 0 && total_q >= 0 && max_q >= 0 && route_rows >= 0, RECACHE_EINVAL,
+  RC_REQUIRE(n_requests >= 0 && total_q >= 0 && max_q >= 0 && route_rows >= 0 && conv_rows >= 0, RECACHE_EINVAL,
              "prefill: negative size");
   RC_REQUIRE(out_dtype_ok(ctx, out_dtype), RECACHE_EINVAL, "prefill: out_dtype must be f32 or the context dtype");
   if (n_requests == 0 || total_q == 0) return RECACHE_OK;
@@ -253,13 +253,40 @@ recache_status recache_attend_prefill(recache_ctx* ctx, const void* q, const voi
   cudaStream_t st = (cudaStream_t)stream;
   RC_CUDA(cudaSetDevice(ctx->device), "prefill: set device");
 
-  RopeStoreArgs ra{k_conv, v_conv, k_conv_out, v_conv_out, cu_q, n_requests, total_q, nullptr, q_pos0,
-                   (int64_t)total_q, 1};
+  RopeStoreArgs ra{k_conv, v_conv, k_conv_out, v_conv_out, cu_q, n_requests, total_q, conv_slot, q_pos0,
+                   conv_rows, conv_slot ? 2 : 1};
+  ra.hist = hist_len;
   RC_CUDA(rc_launch_rope_store(ctx, ra, st), "prefill: rope/store launch");
   PrefillArgs pa{q, out_o, out_dtype, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
-                 route_rows, k_conv_out, v_conv_out, workspace, workspace_bytes};
+                 route_rows, k_conv_out, v_conv_out, workspace, workspace_bytes, conv_rows, conv_slot, hist_len};
   RC_CUDA(rc_launch_prefill_attn(ctx, pa, st), "prefill: attention launch");
   return RECACHE_OK;
+}
+
+recache_status recache_attend_prefill(recache_ctx* ctx, const void* q, const void* k_conv, const void* v_conv,
+                                      const int32_t* cu_q, const int32_t* q_pos0, int32_t n_requests,
+                                      int32_t total_q, int32_t max_q, const void* k_route, const void* v_route,
+                                      const int32_t* route_cu, int64_t route_rows, void* k_conv_out,
+                                      void* v_conv_out, void* out_o, int32_t out_dtype, void* workspace,
+                                      int64_t workspace_bytes, void* stream) {
+  return prefill_impl(ctx, q, k_conv, v_conv, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
+                      route_rows, k_conv_out, v_conv_out, (int64_t)total_q, nullptr, nullptr, out_o, out_dtype,
+                      workspace, workspace_bytes, stream);
+}
+
+recache_status recache_attend_prefill_history(recache_ctx* ctx, const void* q, const void* k_conv, const void* v_conv,
+                                              const int32_t* cu_q, const int32_t* q_pos0, int32_t n_requests,
+                                              int32_t total_q, int32_t max_q, const void* k_route,
+                                              const void* v_route, const int32_t* route_cu, int64_t route_rows,
+                                              void* k_conv_cache, void* v_conv_cache, int64_t cache_rows,
+                                              const int32_t* conv_slot, const int32_t* hist_len, void* out_o,
+                                              int32_t out_dtype, void* workspace, int64_t workspace_bytes,
+                                              void* stream) {
+  if (!ctx) return RECACHE_EINVAL;
+  RC_REQUIRE(conv_slot && hist_len, RECACHE_EINVAL, "prefill_history: null conv_slot / hist_len");
+  return prefill_impl(ctx, q, k_conv, v_conv, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
+                      route_rows, k_conv_cache, v_conv_cache, cache_rows, conv_slot, hist_len, out_o, out_dtype,
+                      workspace, workspace_bytes, stream);
 }
 
 recache_status recache_attend_decode(recache_ctx* ctx, const void* q, const int32_t* q_pos, int32_t batch,

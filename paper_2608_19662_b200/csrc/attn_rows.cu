@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
     const int32_t* __restrict__ pos0, const int32_t* __restrict__ slot,
     const T* __restrict__ k_self, const T* __restrict__ v_self, int64_t self_rows,
     const T* __restrict__ k_route, const T* __restrict__ v_route, const int32_t* __restrict__ route_cu,
-    int prefix_len, int Hq, int G, const float* __restrict__ cos_tab, const float* __restrict__ sin_tab, int max_pos,
+    int prefix_len, const int32_t* __restrict__ hist, int Hq, int G, const float* __restrict__ cos_tab, const float* __restrict__ sin_tab, int max_pos,
     float scale, int32_t* status) {
   __shared__ float q_s[WARPS][D];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -64,8 +64,9 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
   if (t >= cu[n_seq] || j < 0) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_SEQLENS); return; }
   const int pos = (pos0 ? pos0[b] : 0) + j;
   const int64_t base = slot ? (int64_t)slot[b] : (int64_t)cu[b];
+  const int H = hist ? hist[b] : 0;      // earlier-turn rows at the start of the self part, all visible
   if (pos < 0 || pos >= max_pos) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_POS); return; }
-  if (base < 0 || base + j >= self_rows) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_SLOT); return; }
+  if (base < 0 || H < 0 || base + H + j >= self_rows) { if (lane == 0) rc_set_status(status, RECACHE_DEV_BAD_SLOT); return; }
 
   // rotate the query row into shared memory
   constexpr int HALF = D / 2;
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
     } else {
       kb = k_self + ((int64_t)g * self_rows + base) * D;
       vb = v_self + ((int64_t)g * self_rows + base) * D;
-      n = j + 1;
+      n = H + j + 1;
     }
     for (int k0 = 0; k0 < n; k0 += 32) {
       const int kk = k0 + lane;
@@ -140,7 +141,7 @@ cudaError_t launch(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t s
   const float scale = (float)(1.0 / sqrt((double)d));
   RcLaunchScope scope(ctx, a.route_cu ? RC_K_PREFILL_ATTN : RC_K_ENCODE_ATTN, st);
 #define RC_ARGS (const T*)a.q, (TO*)a.o, a.cu, a.n_seq, a.total, a.pos0, a.slot, (const T*)a.k_self, \
-    (const T*)a.v_self, a.self_rows, (const T*)a.k_route, (const T*)a.v_route, a.route_cu, a.prefix_len, Hq, G, \
+    (const T*)a.v_self, a.self_rows, (const T*)a.k_route, (const T*)a.v_route, a.route_cu, a.prefix_len, a.hist, Hq, G, \
     ctx->cos_tab, ctx->sin_tab, ctx->desc.max_pos, scale, ctx->status
   if (d == 64) attn_rows_kernel<T, TO, 64><<<blocks, WARPS * 32, 0, st>>>(RC_ARGS);
   else         attn_rows_kernel<T, TO, 128><<<blocks, WARPS * 32, 0, st>>>(RC_ARGS);

@@ -63,7 +63,7 @@ constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long i
 
 struct TcParams {
   const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter
-  const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu;
+  const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu; const int32_t* hist;
   int n_seq, G, Hq, s;
   int prefix_len;   // > 0: every sequence sees rows g*prefix_len .. of the "route" tensors (shared prefix)
   int64_t self_rows;
@@ -257,10 +257,11 @@ __global__ void __launch_bounds__(1024) tile_plan_kernel(const int32_t* __restri
 struct Item {
   int n_tiles;      // -1: no more work
   int g, seq0, L, tok0, kv_end, pos0, rA0, lenA, nA, b_valid;
+  int H;            // rows that precede the sequence's own tokens in the self part (earlier turns), all visible
   int64_t base;
 };
 enum { IT_NTILES = 0, IT_G, IT_SEQ0, IT_L, IT_TOK0, IT_KVEND, IT_POS0, IT_RA0, IT_LENA, IT_NA, IT_BVALID, IT_BASE_LO,
-       IT_BASE_HI, IT_WORDS = 16 };
+       IT_BASE_HI, IT_H, IT_WORDS = 16 };
 
 // Work index w -> item; false when the caller's index arrays are inconsistent
 // (flagged in the status word; the scheduler skips the item).
@@ -273,7 +274,8 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
   it.L = p.cu[b + 1] - it.seq0;
   it.tok0 = e.y * 2 * TQ;
   it.b_valid = it.tok0 + TQ < it.L;
-  it.kv_end = min(it.L, it.tok0 + 2 * TQ);
+  it.H = p.hist ? p.hist[b] : 0;
+  it.kv_end = it.H + min(it.L, it.tok0 + 2 * TQ);   // self rows the pair can see: the history, then its causal range
   it.base = p.slot ? (int64_t)p.slot[b] : (int64_t)it.seq0;
   it.pos0 = p.pos0 ? p.pos0[b] : 0;
   it.rA0 = 0; it.lenA = 0;
@@ -281,8 +283,8 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
   else if (p.prefix_len > 0) { it.rA0 = it.g * p.prefix_len; it.lenA = p.prefix_len; }
   it.nA = (it.lenA + TILE_N - 1) / TILE_N;
   it.n_tiles = it.nA + (it.kv_end + TILE_N - 1) / TILE_N;
-  const bool ok = it.L > 0 && it.tok0 < it.L && it.lenA >= 0 && it.rA0 >= 0 && it.base >= 0 &&
-                  it.base + it.L <= p.self_rows && it.seq0 >= 0;
+  const bool ok = it.L > 0 && it.tok0 < it.L && it.lenA >= 0 && it.rA0 >= 0 && it.base >= 0 && it.H >= 0 &&
+                  it.base + it.H + it.L <= p.self_rows && it.seq0 >= 0;
   if (!ok) rc_set_status(p.status, RECACHE_DEV_BAD_SLOT);
   return ok;
 }
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const volatile int* r = item_ring + sl * IT_WORDS;
     it.n_tiles = r[IT_NTILES]; it.g = r[IT_G]; it.seq0 = r[IT_SEQ0]; it.L = r[IT_L]; it.tok0 = r[IT_TOK0];
     it.kv_end = r[IT_KVEND]; it.pos0 = r[IT_POS0]; it.rA0 = r[IT_RA0]; it.lenA = r[IT_LENA]; it.nA = r[IT_NA];
-    it.b_valid = r[IT_BVALID];
+    it.b_valid = r[IT_BVALID]; it.H = r[IT_H];
     it.base = (int64_t)(((uint64_t)(uint32_t)r[IT_BASE_HI] << 32) | (uint32_t)r[IT_BASE_LO]);
     if (*abort_flag) it.n_tiles = -1;
     if (release) mbar_arrive(bar(B_IEMPTY + sl));
@@ -377,6 +379,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         if (it.n_tiles > 0) {
           r[IT_G] = it.g; r[IT_SEQ0] = it.seq0; r[IT_L] = it.L; r[IT_TOK0] = it.tok0; r[IT_KVEND] = it.kv_end;
           r[IT_POS0] = it.pos0; r[IT_RA0] = it.rA0; r[IT_LENA] = it.lenA; r[IT_NA] = it.nA; r[IT_BVALID] = it.b_valid;
+          r[IT_H] = it.H;
           r[IT_BASE_LO] = (int)(uint32_t)(it.base & 0xffffffffll); r[IT_BASE_HI] = (int)(uint32_t)((uint64_t)it.base >> 32);
         }
         mbar_arrive(bar(B_IFULL + sl));
@@ -457,7 +460,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_IEMPTY + (item_n & 1u)));
       if (it.n_tiles < 0) break;
-      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, L = it.L, kv_end = it.kv_end;
+      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, L = it.H + it.L, kv_end = it.kv_end;
       const bool b_valid = it.b_valid != 0;
       mbar_wait(bar(B_QREADY), item_n & 1u, abort_flag, p.status);
       mbar_wait(bar(B_KFULL + kv_n % NSTAGE), (kv_n / NSTAGE) & 1u, abort_flag, p.status);
@@ -584,7 +587,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       const bool active = x == 0 || it.b_valid;
       const int t_row = it.tok0 + x * TQ + row / s;     // token (local index)
       const int t_eff = min(t_row, it.L - 1);
-      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA;
+      const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, H = it.H;
       float m_ref = -INFINITY, l_sum = 0.f;
       if (active) {
         for (int i = 0; i < n_tiles; ++i, ++cnt) {
@@ -594,7 +597,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           TMEM_LD32(t_s + 0, sr, 0); TMEM_LD32(t_s + 32, sr, 32); TMEM_LD32(t_s + 64, sr, 64); TMEM_LD32(t_s + 96, sr, 96);
           tmem_wait_ld();
           // keys this row may see in this tile: columns [0, lim)
-          const int lim = i < nA ? lenA - i * TILE_N : t_eff - (i - nA) * TILE_N + 1;
+          const int lim = i < nA ? lenA - i * TILE_N : H + t_eff - (i - nA) * TILE_N + 1;
           if (lim < TILE_N) {
 #pragma unroll
             for (int c = 0; c < 128; ++c) if (c >= lim) sr[c] = 0xff800000u;   // -inf
@@ -791,6 +794,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   p.items = items; p.header = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
   p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.out = a.o;
   p.prefix_len = a.route_cu ? 0 : a.prefix_len;
+  p.hist = a.hist;
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)ctx->desc.head_dim));
   p.status = ctx->status;

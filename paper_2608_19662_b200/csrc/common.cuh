@@ -78,14 +78,16 @@ template <> __device__ __forceinline__ __nv_bfloat16 rc_from_float<__nv_bfloat16
 //  mode 0 (encode): token t of resource i -> position pos0[i] + t - cu[i] (pos0 may be null = 0),
 //                   row slot[i] + (t - cu[i])
 //  mode 1 (prefill): token t of request b -> position pos0[b] + (t - cu[b]), row t
+//  mode 2 (prefill into a conversation cache): same position, row slot[b] + hist[b] + (t - cu[b])
 struct RopeStoreArgs {
   const void* k; const void* v;       // [total][G][d]
   void* k_dst; void* v_dst;           // [G][dst_rows][d]
   const int32_t* cu; int n_seq; int total;
-  const int32_t* slot;                // mode 0
-  const int32_t* pos0;                // mode 1; optional in mode 0
+  const int32_t* slot;                // mode 0, 2
+  const int32_t* pos0;                // mode 1, 2; optional in mode 0
   int64_t dst_rows;
   int mode;
+  const int32_t* hist = nullptr;      // mode 2: rows already in each sequence's region; new rows follow them
 };
 cudaError_t rc_launch_rope_store(const recache_ctx* ctx, const RopeStoreArgs& a, cudaStream_t st);
 
@@ -100,6 +102,7 @@ struct AttnRowsArgs {
   int64_t self_rows;
   const void* k_route; const void* v_route; const int32_t* route_cu;  // null for encode
   int prefix_len;   // > 0 (with route_cu null): every sequence sees rows g*prefix_len .. +prefix_len of k_route/v_route
+  const int32_t* hist = nullptr;   // rows that precede each sequence's own tokens in the self part, all visible
 };
 cudaError_t rc_launch_attn_rows(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t st);
 
@@ -143,8 +146,11 @@ struct PrefillArgs {
   const void* q; void* o; int out_dtype;
   const int32_t* cu_q; const int32_t* pos0; int n_req; int total_q; int max_q;
   const void* k_route; const void* v_route; const int32_t* route_cu; int64_t route_rows;
-  const void* k_conv; const void* v_conv;   // rotated, [G][total_q][d]
+  const void* k_conv; const void* v_conv;   // rotated, [G][conv_rows][d]
   void* workspace; int64_t workspace_bytes;
+  int64_t conv_rows;                        // rows per group of k_conv / v_conv
+  const int32_t* conv_slot = nullptr;       // first row of each request's region (null: cu_q[b])
+  const int32_t* hist = nullptr;            // earlier-turn rows at the start of that region (null: 0)
 };
 int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, int max_len);
 int64_t rc_prefill_workspace_bytes(const recache_ctx* ctx, int n_req, int total_q, int max_q);
@@ -163,6 +169,7 @@ struct TcAttnArgs {
   const void* k_route; const void* v_route; const int32_t* route_cu; int64_t route_rows;
   void* workspace;
   int prefix_len;   // > 0 (route_cu null): all sequences see rows g*prefix_len .. of k_route/v_route ([G*prefix_len][128])
+  const int32_t* hist = nullptr;   // rows preceding each sequence's own tokens in the self part (earlier turns), all visible
 };
 bool rc_tc_supported(const recache_ctx* ctx);
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);

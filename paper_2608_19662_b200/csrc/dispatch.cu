@@ -29,12 +29,12 @@ cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, c
 
 cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a, cudaStream_t st) {
   if (rc_tc_supported(ctx)) {
-    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.max_q, a.pos0, nullptr, a.k_conv, a.v_conv,
-                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace, 0};
+    TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.max_q, a.pos0, a.conv_slot, a.k_conv, a.v_conv,
+                 a.conv_rows, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace, 0, a.hist};
     return rc_launch_attn_tc(ctx, t, st);
   }
-  AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, nullptr, a.k_conv, a.v_conv,
-                 (int64_t)a.total_q, a.k_route, a.v_route, a.route_cu, 0};
+  AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, a.conv_slot, a.k_conv, a.v_conv,
+                 a.conv_rows, a.k_route, a.v_route, a.route_cu, 0, a.hist};
   return rc_launch_attn_rows(ctx, r, st);
 }
 

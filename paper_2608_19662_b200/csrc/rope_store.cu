@@ -50,7 +50,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) rope_store_kernel(
     const T* __restrict__ k, const T* __restrict__ v, T* __restrict__ k_dst, T* __restrict__ v_dst,
     const int32_t* __restrict__ cu, int n_seq, int total, const int32_t* __restrict__ slot,
-    const int32_t* __restrict__ pos0, int64_t dst_rows, int mode, int G, int d,
+    const int32_t* __restrict__ pos0, const int32_t* __restrict__ hist, int64_t dst_rows, int mode, int G, int d,
     const float* __restrict__ cos_tab, const float* __restrict__ sin_tab, int max_pos,
     int32_t* status) {
   constexpr int N = Vec16<T>::N;
@@ -68,7 +68,8 @@ __global__ void __launch_bounds__(256) rope_store_kernel(
   // position = the sequence's first position (0 when none is given) + index inside the sequence;
   // row = the sequence's first cache row + that index (encode) or the token index itself (prefill)
   const int pos = (pos0 ? pos0[b] : 0) + local;
-  const int64_t row = mode == 0 ? (int64_t)slot[b] + local : (int64_t)t;
+  const int64_t row = mode == 0 ? (int64_t)slot[b] + local
+                    : mode == 2 ? (int64_t)slot[b] + (hist ? hist[b] : 0) + local : (int64_t)t;
   if (t >= cu[n_seq] || cu[b + 1] < cu[b]) { rc_set_status(status, RECACHE_DEV_BAD_SEQLENS); return; }
   if (row < 0 || row >= dst_rows) { rc_set_status(status, RECACHE_DEV_BAD_SLOT); return; }
   if (pos < 0 || pos >= max_pos) { rc_set_status(status, RECACHE_DEV_BAD_POS); return; }
@@ -114,12 +115,12 @@ cudaError_t rc_launch_rope_store(const recache_ctx* ctx, const RopeStoreArgs& a,
   if (bf)
     rope_store_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
         (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v, (__nv_bfloat16*)a.k_dst, (__nv_bfloat16*)a.v_dst,
-        a.cu, a.n_seq, a.total, a.slot, a.pos0, a.dst_rows, a.mode, G, d, ctx->cos_tab, ctx->sin_tab,
+        a.cu, a.n_seq, a.total, a.slot, a.pos0, a.hist, a.dst_rows, a.mode, G, d, ctx->cos_tab, ctx->sin_tab,
         ctx->desc.max_pos, ctx->status);
   else
     rope_store_kernel<float><<<blocks, threads, 0, st>>>(
         (const float*)a.k, (const float*)a.v, (float*)a.k_dst, (float*)a.v_dst,
-        a.cu, a.n_seq, a.total, a.slot, a.pos0, a.dst_rows, a.mode, G, d, ctx->cos_tab, ctx->sin_tab,
+        a.cu, a.n_seq, a.total, a.slot, a.pos0, a.hist, a.dst_rows, a.mode, G, d, ctx->cos_tab, ctx->sin_tab,
         ctx->desc.max_pos, ctx->status);
   return cudaGetLastError();
 }

@@ -488,3 +488,21 @@ def test_block_variant_no_cross_resource_attention_with_global_positions():
     o_local, _, _ = orc.encode_resources(q, k, v, cu, sh.rope_theta, pos_offset=[P] * 3, prefix_k=pk, prefix_v=pv)
     assert np.abs(o_local - o)[cu[1]:].max() > 1e-3                # offsets do matter once there is a prefix
     assert np.allclose(o_local[:cu[1]], o[:cu[1]], atol=1e-12)     # ... except for the first resource (same offset)
+
+
+# ------------------------------------------------------- multi-turn history --
+def test_second_turn_with_history_equals_rows_of_one_long_prefill():
+    """Turn 1 (20 tokens) then turn 2 (12 tokens) with turn 1 as all-visible
+    history, positions continuing, gives the turn-2 rows of a single 32-token
+    prefill (already pinned against brute force)."""
+    pool, req, kc, vc, rows = _c1_pipeline()
+    sh = pool.shape
+    q, k, v = f64(req.q), f64(req.k_conv), f64(req.v_conv)
+    o_all, kh_all = orc.attend_prefill(q, k, v, req.cu_q, req.q_pos0, rows, kc, vc, sh.rope_theta)
+    n1 = 20
+    o1, kh1 = orc.attend_prefill(q[:n1], k[:n1], v[:n1], [0, n1], [64], rows, kc, vc, sh.rope_theta)
+    assert np.allclose(o1, o_all[:n1], atol=1e-12)
+    hist_k = [np.transpose(kh1, (1, 0, 2))]; hist_v = [np.transpose(v[:n1], (1, 0, 2))]
+    o2, _ = orc.attend_prefill(q[n1:], k[n1:], v[n1:], [0, 32 - n1], [64 + n1], rows, kc, vc, sh.rope_theta,
+                               hist_k=hist_k, hist_v=hist_v)
+    assert np.allclose(o2, o_all[n1:], atol=1e-12)
