@@ -39,6 +39,12 @@ sys.path.insert(0, ROOT)
 
 from paper_2608_19662_b200 import workloads as wl  # noqa: E402
 
+# DRAM traffic of the encode attention launch, from the ncu capture summarised in
+# profiles/attn_tc_medium_case.md (dram__bytes_read.sum + dram__bytes_write.sum = 408.3 MB for 21,626
+# resource tokens).  The full workload is too large for a multi-pass capture; traffic grows in proportion
+# to the tokens (Q read, O written, K/V read once from HBM and re-read from L2), so it is scaled per token.
+NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 408.347e6 / 21626
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -409,7 +415,9 @@ def main():
     ach = w.flops["encode"] / (enc_ms * 1e-3) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {"kernel": "encode_attn", "bound": "tensor", "achieved": ach, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": ach / peak_tf, "traffic": None, "peak_source": f"{peak_src} (sustained bf16)",
+                "frac": ach / peak_tf, "traffic": NCU_ENCODE_DRAM_BYTES_PER_TOKEN * w.pool.total_tokens,
+                "traffic_note": "ncu DRAM bytes of a 21,626-token launch scaled per token",
+                "algorithmic_bytes": w.pool.total_tokens * (2 * w.shape.n_q_heads + 2 * w.shape.n_kv_heads) * w.shape.head_dim * 2, "peak_source": f"{peak_src} (sustained bf16)",
                 "flops_per_launch": w.flops["encode"], "ms_per_launch": enc_ms}
     stages = {}
     if "prefill_attn" in per:
