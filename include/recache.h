@@ -188,7 +188,8 @@ RECACHE_API recache_status recache_encode_resources_prefixed(recache_ctx* ctx,
  *   route_cu  [B*G+1]  exclusive prefix of route lengths
  *   route_len [B*G]    (optional, may be NULL) the lengths themselves
  *   route_idx [row_capacity] cache row of every compacted row, packed order
- *   mode RECACHE_PACKED: k_out/v_out [row_capacity][d] packed route KV
+ *   mode RECACHE_PACKED: k_out/v_out [row_capacity][d] packed route KV; both may be
+ *        NULL: indices and prefix only, no row is copied (see recache_attend_decode_gather)
  *   mode RECACHE_PAGED : k_out/v_out are page pools [n_pool_pages][page_tokens][d];
  *        route r takes ceil(len_r / page_tokens) consecutive entries of
  *        free_pages [n_free_pages], starting where route r-1 stopped; row n of
@@ -272,6 +273,28 @@ RECACHE_API recache_status recache_attend_decode(recache_ctx* ctx,
     const void* k_new, const void* v_new,
     void* k_pages, void* v_pages, int64_t n_pages,
     const int32_t* res_page_table, int32_t max_res_pages, const int32_t* res_len,
+    const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
+ * Routed decode without materialising the resource rows (zero-copy): the
+ * resource part of item it = b * G + g is read straight from the resource cache,
+ * rows route_idx[route_cu[it] .. route_cu[it+1]) of group g - the index list that
+ * recache_compact_routes writes (call it with k_out = v_out = NULL, packed mode,
+ * to get the indices only: no key / value byte is moved, and requests that share
+ * a resource share its cache rows).  History stays paged as in
+ * recache_attend_decode; same softmax, same results.
+ *   max_res_pages: upper bound of ceil(route length / page_tokens), used to size
+ *   the split plan and the workspace (recache_decode_workspace_bytes).
+ * bf16 contexts with head_dim 128 and 64-token pages only.
+ */
+RECACHE_API recache_status recache_attend_decode_gather(recache_ctx* ctx,
+    const void* q, const int32_t* q_pos, int32_t batch,
+    const void* k_new, const void* v_new,
+    const void* k_cache, const void* v_cache, int64_t pool_tokens,
+    const int32_t* route_idx, const int32_t* route_cu, int32_t max_res_pages,
+    void* k_pages, void* v_pages, int64_t n_pages,
     const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
     void* out_o, int32_t out_dtype,
     void* workspace, int64_t workspace_bytes, void* stream);

@@ -55,6 +55,8 @@ SIGNATURES = {
                                                  _I64, _P, _P, _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                         _P, _I32, _P, _I64, _P]),
+    "recache_attend_decode_gather": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _P, _I32, _P, _P, _I64,
+                                               _P, _I32, _P, _P, _I32, _P, _I64, _P]),
     "recache_build_routes": (C.c_int, [C.POINTER(C.c_double), _I32, C.POINTER(C.c_double), _I32, _I32, _I32,
                                        C.POINTER(C.c_uint8), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                        C.POINTER(C.c_double)]),
@@ -231,7 +233,8 @@ class ReCache:
         st = self.lib.recache_compact_routes(
             self.h, _ptr(k_cache), _ptr(v_cache), k_cache.shape[1], _ptr(keep), _ptr(res_off), _ptr(res_slot),
             _ptr(res_len), n_req, total_listed, _ptr(vis), mode, _ptr(route_cu), _ptr(route_len), _ptr(route_idx),
-            route_idx.numel() if paged else min(route_idx.numel(), k_out.shape[0]), _ptr(k_out), _ptr(v_out),
+            route_idx.numel() if (paged or k_out is None) else min(route_idx.numel(), k_out.shape[0]), _ptr(k_out),
+            _ptr(v_out),
             _ptr(page_table),
             page_table.shape[1] if paged else 0, _ptr(free_pages), free_pages.numel() if paged else 0,
             k_out.shape[0] if paged else 0, _ptr(ws), ws.numel(), _stream())
@@ -289,6 +292,23 @@ class ReCache:
                                             _ptr(res_len), _ptr(hist_page_table), mh, _ptr(hist_len), _ptr(out), oc,
                                             _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_attend_decode")
+        return out
+
+    def attend_decode_gather(self, q, q_pos, k_cache, v_cache, route_idx, route_cu, max_res_pages, k_pages, v_pages,
+                             hist_page_table, hist_len, k_new=None, v_new=None, out=None, out_dtype=None, workspace=None):
+        """recache_attend_decode_gather: decode whose resource rows are read from the cache through the
+        compaction's index list (nothing materialised).  Returns o [B,Hq,d]."""
+        batch = q.shape[0]
+        od, oc = self._out_code(out_dtype)
+        if out is None:
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        mh = hist_page_table.shape[1]
+        ws = workspace if workspace is not None else self.workspace(self.decode_workspace_bytes(batch, max_res_pages, mh))
+        st = self.lib.recache_attend_decode_gather(
+            self.h, _ptr(q), _ptr(q_pos), batch, _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), k_cache.shape[1],
+            _ptr(route_idx), _ptr(route_cu), int(max_res_pages), _ptr(k_pages), _ptr(v_pages), k_pages.shape[0],
+            _ptr(hist_page_table), mh, _ptr(hist_len), _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
+        self._check(st, "recache_attend_decode_gather")
         return out
 
     def attend_decode_noalloc(self, q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page_table, hist_len,

@@ -212,9 +212,12 @@ recache_status recache_compact_routes(recache_ctx* ctx, const void* k_cache, con
              "compact: negative size");
   RC_REQUIRE(mode == RECACHE_PACKED || mode == RECACHE_PAGED, RECACHE_EINVAL, "compact: bad mode");
   RC_REQUIRE(route_cu && res_off, RECACHE_EINVAL, "compact: null route_cu / res_off");
-  if (total_listed > 0)
-    RC_REQUIRE(k_cache && v_cache && keep && res_slot && res_len && vis && route_idx && k_out && v_out,
-               RECACHE_EINVAL, "compact: null pointer");
+  if (total_listed > 0) {
+    RC_REQUIRE(keep && res_slot && res_len && vis && route_idx, RECACHE_EINVAL, "compact: null pointer");
+    RC_REQUIRE((k_out == nullptr) == (v_out == nullptr), RECACHE_EINVAL, "compact: k_out and v_out go together");
+    RC_REQUIRE(!k_out || (k_cache && v_cache), RECACHE_EINVAL, "compact: null cache");
+    RC_REQUIRE(k_out || mode == RECACHE_PACKED, RECACHE_EINVAL, "compact: index-only compaction is a packed-mode call");
+  }
   if (mode == RECACHE_PAGED)
     RC_REQUIRE(page_table && free_pages && max_pages_per_route > 0 && n_free_pages >= 0 && n_pool_pages > 0,
                RECACHE_EINVAL, "compact: paged mode needs page_table, free_pages and pool sizes");
@@ -314,6 +317,38 @@ recache_status recache_attend_decode(recache_ctx* ctx, const void* q, const int3
                hist_page_table, max_hist_pages, hist_len, out_o, out_dtype, workspace, workspace_bytes};
   if (k_new) RC_CUDA(rc_launch_decode_append(ctx, a, st), "decode: append launch");
   RC_CUDA(rc_launch_decode(ctx, a, st), "decode: attention launch");
+  return RECACHE_OK;
+}
+
+recache_status recache_attend_decode_gather(recache_ctx* ctx, const void* q, const int32_t* q_pos, int32_t batch,
+                                            const void* k_new, const void* v_new, const void* k_cache,
+                                            const void* v_cache, int64_t pool_tokens, const int32_t* route_idx,
+                                            const int32_t* route_cu, int32_t max_res_pages, void* k_pages,
+                                            void* v_pages, int64_t n_pages, const int32_t* hist_page_table,
+                                            int32_t max_hist_pages, const int32_t* hist_len, void* out_o,
+                                            int32_t out_dtype, void* workspace, int64_t workspace_bytes,
+                                            void* stream) {
+  if (!ctx) return RECACHE_EINVAL;
+  RC_REQUIRE(batch >= 0 && n_pages >= 0 && max_res_pages >= 0 && max_hist_pages > 0 && pool_tokens >= 0,
+             RECACHE_EINVAL, "decode_gather: bad size");
+  RC_REQUIRE(out_dtype_ok(ctx, out_dtype), RECACHE_EINVAL, "decode_gather: out_dtype must be f32 or the context dtype");
+  RC_REQUIRE(rc_decode_split_supported(ctx), RECACHE_EUNSUPPORTED,
+             "decode_gather: needs a bf16 context with head_dim 128 and 64-token pages");
+  if (batch == 0) return RECACHE_OK;
+  RC_REQUIRE(q && q_pos && k_cache && v_cache && route_idx && route_cu && k_pages && v_pages && hist_page_table &&
+                 hist_len && out_o, RECACHE_EINVAL, "decode_gather: null pointer");
+  RC_REQUIRE((k_new == nullptr) == (v_new == nullptr), RECACHE_EINVAL, "decode_gather: k_new and v_new go together");
+  RC_REQUIRE(aligned16(q) && aligned16(k_cache) && aligned16(v_cache) && aligned16(k_pages) && aligned16(v_pages) &&
+                 aligned16(out_o), RECACHE_EINVAL, "decode_gather: tensors must be 16-byte aligned");
+  const int64_t need = rc_decode_workspace_bytes(ctx, batch, max_res_pages, max_hist_pages);
+  RC_REQUIRE(need == 0 || (workspace && workspace_bytes >= need), RECACHE_ENOMEM, "decode_gather: workspace too small");
+  cudaStream_t st = (cudaStream_t)stream;
+  RC_CUDA(cudaSetDevice(ctx->device), "decode_gather: set device");
+  DecodeArgs a{q, q_pos, batch, k_new, v_new, k_pages, v_pages, n_pages, nullptr, max_res_pages, nullptr,
+               hist_page_table, max_hist_pages, hist_len, out_o, out_dtype, workspace, workspace_bytes};
+  a.k_cache = k_cache; a.v_cache = v_cache; a.pool_tokens = pool_tokens; a.route_idx = route_idx; a.route_cu = route_cu;
+  if (k_new) RC_CUDA(rc_launch_decode_append(ctx, a, st), "decode_gather: append launch");
+  RC_CUDA(rc_launch_decode_split(ctx, a, st), "decode_gather: attention launch");
   return RECACHE_OK;
 }
 

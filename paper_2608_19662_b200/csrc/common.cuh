@@ -129,6 +129,10 @@ struct DecodeArgs {
   const int32_t* hist_pt; int max_hist_pages; const int32_t* hist_len;
   void* o; int out_dtype;
   void* workspace; int64_t workspace_bytes;
+  // gather variant (route_idx != null): the resource part of item `it` is rows
+  // route_idx[route_cu[it] .. route_cu[it+1]) of the cache; res_pt / res_len are unused
+  const void* k_cache = nullptr; const void* v_cache = nullptr; int64_t pool_tokens = 0;
+  const int32_t* route_idx = nullptr; const int32_t* route_cu = nullptr;
 };
 cudaError_t rc_launch_decode_append(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
 cudaError_t rc_launch_decode_rows(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);

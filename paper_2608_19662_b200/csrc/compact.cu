@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(TPB) compact_gather_kernel(
     }
     __syncthreads();
     // with few (resource, group) pairs the copy is shared by gridDim.z CTAs that all ran the (cheap) scan
-    const int n_piece = tot * segs;
+    const int n_piece = k_out ? tot * segs : 0;   // index-only compaction moves no rows
     for (int e0 = threadIdx.x + blockIdx.z * TPB * 4; e0 < n_piece; e0 += TPB * 4 * gridDim.z) {
       uint4 kx[4], vx[4];
       int64_t dof[4];

@@ -31,16 +31,28 @@ constexpr int NSTAGE = 6;
 constexpr int PAGE_BYTES = PT * D * 2; // 16 KB
 constexpr int BOX_BYTES = 8192;        // [64 tokens][64 bf16], 128-byte swizzle
 constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+// Gather variant: the resource rows of a chunk come straight from the cache with 16-byte cp.async
+// copies (half a warp per 256-byte row) written at the swizzled positions a TMA page load would use,
+// so the consumers see one layout.  Four producer warps share a chunk (16 rows each): one warp alone
+// cannot issue the 2048 copies of a chunk fast enough.  A full barrier then takes 128 arrivals: every
+// producer lane's copies (gathered chunk), or the expect-tx arrival plus 127 plain ones (TMA page).
 constexpr int NCW = 3;                 // consumer warps; NSTAGE % NCW == 0
 static_assert(NSTAGE % NCW == 0, "a stage must always be consumed by the same warp");
+constexpr int NPW_GATHER = 4;           // producer warps of the gather variant (the paged variant has one)
 constexpr int NTHREADS = (NCW + 1) * 32;
+constexpr int NTHREADS_GATHER = (NCW + NPW_GATHER) * 32;
 constexpr int SM_STAGES = 0;
-constexpr int SM_BAR = NSTAGE * STAGE_BYTES;          // full[NSTAGE], empty[NSTAGE]
-constexpr int SM_Q = SM_BAR + 2 * NSTAGE * 8 + 32;    // per-warp rotated q: NCW x 8 x 128 bf16
-constexpr int SM_MERGE = SM_Q + NCW * 8 * D * 2;      // NCW x 8 x (2 + 128) floats
-constexpr int SM_MISC = SM_MERGE + NCW * 8 * 130 * 4;
-constexpr int SM_TOTAL = SM_MISC + 64;
-constexpr int SM_ALLOC = SM_TOTAL + 1024;
+template <bool GATHER> struct Lay {
+  static constexpr int STAGE = STAGE_BYTES;
+  static constexpr int VOFF = PAGE_BYTES;                               // V half inside a stage
+  static constexpr int BAR = NSTAGE * STAGE;                            // full[NSTAGE], empty[NSTAGE]
+  static constexpr int Q = BAR + 2 * NSTAGE * 8 + 32;                   // per-warp rotated q: NCW x 8 x 128 bf16
+  static constexpr int MERGE = Q + NCW * 8 * D * 2;                     // NCW x 8 x (2 + 128) floats
+  static constexpr int MISC = MERGE + NCW * 8 * 130 * 4;
+  static constexpr int TOTAL = MISC + 64;
+  static constexpr int ALLOC = TOTAL + 1024;
+};
+static_assert(Lay<true>::ALLOC <= 232448, "shared memory");
 constexpr long long WAIT_CYCLES = 4000000000ll;
 
 struct DecParams {
@@ -53,6 +65,9 @@ struct DecParams {
   const float* cos_tab; const float* sin_tab; int max_pos;
   float scale_log2;
   int32_t* status;
+  // gather variant: the resource part of item `it` is rows route_idx[route_cu[it] .. route_cu[it+1]) of the cache
+  const __nv_bfloat16* k_cache; const __nv_bfloat16* v_cache; int64_t pool_tokens;
+  const int32_t* route_idx; const int32_t* route_cu;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -87,6 +102,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)) : "memory");
+}
+// the barrier gets one (pre-counted) arrival when all earlier cp.async of this thread have landed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
@@ -112,11 +134,12 @@ __device__ __forceinline__ void bar_consumers() { asm volatile("bar.sync 1, %0;"
 
 // Pages of item `it` and the range split `sp` owns.
 struct UnitPages { int n_res_pages, n_hist_pages, p0, p1, res_len, hist_len; };
+template <bool GATHER>
 __device__ __forceinline__ UnitPages unit_pages(const DecParams& p, int it, int sp) {
   UnitPages u;
-  u.res_len = max(p.res_len[it], 0);
+  u.res_len = GATHER ? max(p.route_cu[it + 1] - p.route_cu[it], 0) : max(p.res_len[it], 0);
   u.hist_len = max(p.hist_len[it], 0);
-  u.n_res_pages = min((u.res_len + PT - 1) / PT, p.max_res_pages);
+  u.n_res_pages = GATHER ? (u.res_len + PT - 1) / PT : min((u.res_len + PT - 1) / PT, p.max_res_pages);
   u.n_hist_pages = min((u.hist_len + PT - 1) / PT, p.max_hist_pages);
   const int total = u.n_res_pages + u.n_hist_pages;
   u.p0 = (int)((int64_t)total * sp / p.n_splits);
@@ -124,13 +147,15 @@ __device__ __forceinline__ UnitPages unit_pages(const DecParams& p, int it, int 
   return u;
 }
 
-template <typename TO>
-__global__ void __launch_bounds__(NTHREADS, 1) decode_split_kernel(const __grid_constant__ CUtensorMap tm_k,
+template <typename TO, bool GATHER>
+__global__ void __launch_bounds__(GATHER ? NTHREADS_GATHER : NTHREADS, 1) decode_split_kernel(const __grid_constant__ CUtensorMap tm_k,
                                                                    const __grid_constant__ CUtensorMap tm_v,
                                                                    const DecParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t sm = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sm_gen = smem_raw + (sm - smem_u32(smem_raw));
+  using L = Lay<GATHER>;
+  constexpr int SM_BAR = L::BAR, SM_Q = L::Q, SM_MERGE = L::MERGE, SM_MISC = L::MISC, STAGE = L::STAGE, VOFF = L::VOFF;
   const uint32_t bars = sm + SM_BAR;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_gen + SM_MISC);
   auto full = [&](int i) { return bars + 8u * (uint32_t)i; };
@@ -140,34 +165,76 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_split_kernel(const __grid_
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    for (int i = 0; i < NSTAGE; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
+    for (int i = 0; i < NSTAGE; ++i) { mbar_init(full(i), GATHER ? 32 * NPW_GATHER : 1); mbar_init(empty(i), 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  if (warp == NCW) {
-    // ===================== producer =====================
-    if (lane == 0) {
-      uint32_t n = 0;   // pages issued so far (ring position)
-      for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        const int it = unit / p.n_splits, sp = unit % p.n_splits;
-        const UnitPages u = unit_pages(p, it, sp);
-        for (int lp = u.p0; lp < u.p1; ++lp, ++n) {
-          int pg = lp < u.n_res_pages ? p.res_pt[(int64_t)it * p.max_res_pages + lp]
-                                      : p.hist_pt[(int64_t)it * p.max_hist_pages + (lp - u.n_res_pages)];
-          if (pg < 0 || pg >= p.n_pages) { rc_set_status(p.status, RECACHE_DEV_BAD_PAGE); pg = 0; }
-          const int st = n % NSTAGE;
-          mbar_wait(empty(st), ((n / NSTAGE) & 1u) ^ 1u, abort_flag, p.status);
-          mbar_expect_tx(full(st), STAGE_BYTES);
-          const uint32_t dst = sm + SM_STAGES + st * STAGE_BYTES;
-          tma_load_2d(dst, &tm_k, full(st), 0, pg * PT);
-          tma_load_2d(dst + BOX_BYTES, &tm_k, full(st), 64, pg * PT);
-          tma_load_2d(dst + PAGE_BYTES, &tm_v, full(st), 0, pg * PT);
-          tma_load_2d(dst + PAGE_BYTES + BOX_BYTES, &tm_v, full(st), 64, pg * PT);
+  if (warp >= NCW) {
+    // ===================== producer(s) =====================
+    const int pw = warp - NCW;                         // producer warp index (0 in the paged variant)
+    int64_t idx_next = 0;                              // gather variant: row index prefetched for the next chunk
+    uint32_t n = 0;   // pages issued so far (ring position)
+    for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+      const int it = unit / p.n_splits, sp = unit % p.n_splits;
+      const UnitPages u = unit_pages<GATHER>(p, it, sp);
+      for (int lp = u.p0; lp < u.p1; ++lp, ++n) {
+        const int st = n % NSTAGE;
+        const uint32_t dst = sm + SM_STAGES + st * STAGE;
+        if (GATHER && lp < u.n_res_pages) {
+          // 64 route rows straight from the cache: half a warp copies one 256-byte row, 16 bytes per lane
+          const int g = it % p.G;
+          const int r0 = p.route_cu[it] + lp * PT;
+          const int valid = min(PT, u.res_len - lp * PT);
+          constexpr int RPW = PT / NPW_GATHER;                 // rows per producer warp (16)
+          // cache row of chunk row pw * 16 + lane (lanes 0..15): fetched one chunk ahead inside a unit
+          auto load_idx = [&](int chunk) -> int64_t {
+            const int rr = chunk * PT + pw * RPW + lane;
+            return (lane < RPW && rr < u.res_len) ? (int64_t)p.route_idx[p.route_cu[it] + rr] : 0;
+          };
+          int64_t idx_l = (lp == u.p0) ? load_idx(lp) : idx_next;
+          if (lp + 1 < u.p1 && lp + 1 < u.n_res_pages) idx_next = load_idx(lp + 1);
+          if (idx_l < 0 || idx_l >= p.pool_tokens) {
+            rc_set_status(p.status, RECACHE_DEV_BAD_SLOT);
+            idx_l = min(max(idx_l, (int64_t)0), p.pool_tokens - 1);
+          }
+          if (lane == 0) mbar_wait(empty(st), ((n / NSTAGE) & 1u) ^ 1u, abort_flag, p.status);
+          __syncwarp();
+          const int c = lane & 15;
+#pragma unroll
+          for (int rr = 0; rr < RPW; rr += 2) {
+            const int lrow = rr + (lane >> 4);
+            const int row = pw * RPW + lrow;
+            const int64_t idx = __shfl_sync(0xffffffffu, idx_l, lrow);
+            if (row < valid) {
+              const int64_t off = ((int64_t)g * p.pool_tokens + idx) * D + c * 8;
+              const uint32_t d0 = dst + (c >> 3) * BOX_BYTES + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+              cp_async16(d0, p.k_cache + off);
+              cp_async16(d0 + VOFF, p.v_cache + off);
+            }
+          }
+          cp_async_arrive(full(st));
+        } else {
+          if (lane == 0 && pw == 0) {
+            int pg = (!GATHER && lp < u.n_res_pages) ? p.res_pt[(int64_t)it * p.max_res_pages + lp]
+                                                     : p.hist_pt[(int64_t)it * p.max_hist_pages + (lp - u.n_res_pages)];
+            if (pg < 0 || pg >= p.n_pages) { rc_set_status(p.status, RECACHE_DEV_BAD_PAGE); pg = 0; }
+            mbar_wait(empty(st), ((n / NSTAGE) & 1u) ^ 1u, abort_flag, p.status);
+            mbar_expect_tx(full(st), STAGE_BYTES);
+            tma_load_2d(dst, &tm_k, full(st), 0, pg * PT);
+            tma_load_2d(dst + BOX_BYTES, &tm_k, full(st), 64, pg * PT);
+            tma_load_2d(dst + VOFF, &tm_v, full(st), 0, pg * PT);
+            tma_load_2d(dst + VOFF + BOX_BYTES, &tm_v, full(st), 64, pg * PT);
+          }
+          if (GATHER) {           // the other 127 of the 128 arrivals a full barrier takes in this variant
+            if (lane == 0 && pw != 0) mbar_wait(empty(st), ((n / NSTAGE) & 1u) ^ 1u, abort_flag, p.status);
+            __syncwarp();         // (not before this warp has seen the stage released)
+            if (lane != 0 || pw != 0) mbar_arrive(full(st));
+          }
         }
+        __syncwarp();
       }
     }
-    __syncwarp();
   } else {
     // ===================== consumers =====================
     const int gq = lane >> 2, tq = lane & 3;           // fragment row (query head) and column pair
@@ -178,9 +245,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_split_kernel(const __grid_
     for (int unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
       const int it = unit / p.n_splits, sp = unit % p.n_splits;
       const int b = it / p.G, g = it % p.G;
-      const UnitPages u = unit_pages(p, it, sp);
+      const UnitPages u = unit_pages<GATHER>(p, it, sp);
       if (sp == 0 && lane == 0 && warp == 0) {
-        if (u.hist_len < 1 || (u.res_len + PT - 1) / PT > p.max_res_pages || (u.hist_len + PT - 1) / PT > p.max_hist_pages)
+        if (u.hist_len < 1 || (!GATHER && (u.res_len + PT - 1) / PT > p.max_res_pages) ||
+            (u.hist_len + PT - 1) / PT > p.max_hist_pages)
           rc_set_status(p.status, RECACHE_DEV_BAD_PAGE);
       }
       // ---- rotated query heads of the group -> A fragments (rows >= s are zero) ----
@@ -225,10 +293,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_split_kernel(const __grid_
         if (lp < u.n_res_pages) valid = min(PT, u.res_len - lp * PT);
         else valid = min(PT, u.hist_len - (lp - u.n_res_pages) * PT);
         mbar_wait(full(st), (n / NSTAGE) & 1u, abort_flag, p.status);
-        const uint32_t kb = sm + SM_STAGES + st * STAGE_BYTES, vb = kb + PAGE_BYTES;
+        const uint32_t kb = sm + SM_STAGES + st * STAGE, vb = kb + VOFF;
         if (valid < PT) {
           // slots past the end of the part were never written: clear their values (0 * NaN would poison O)
-          uint8_t* vg = sm_gen + SM_STAGES + st * STAGE_BYTES + PAGE_BYTES;
+          uint8_t* vg = sm_gen + SM_STAGES + st * STAGE + VOFF;
           const int v0 = max(valid, 0);
           for (int e = lane; e < (PT - v0) * 16; e += 32) {
             const int r = v0 + (e >> 4), c = e & 15;
@@ -450,19 +518,23 @@ cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, 
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
   p.status = ctx->status;
+  p.k_cache = (const __nv_bfloat16*)a.k_cache; p.v_cache = (const __nv_bfloat16*)a.v_cache;
+  p.pool_tokens = a.pool_tokens; p.route_idx = a.route_idx; p.route_cu = a.route_cu;
   const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
   const unsigned grid = (unsigned)(units < sms ? units : sms);
-  const bool f32 = a.out_dtype == RECACHE_F32;
+  const bool f32 = a.out_dtype == RECACHE_F32, gather = a.route_idx != nullptr;
   {
     RcLaunchScope scope(ctx, RC_K_DECODE_ATTN, st);
-    if (f32) {
-      static bool done = false;
-      if (!done) { cudaFuncSetAttribute(decode_split_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); done = true; }
-      decode_split_kernel<float><<<grid, NTHREADS, SM_ALLOC, st>>>(tk, tv, p);
+    auto launch = [&](auto kernel, int smem) {
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      kernel<<<grid, gather ? NTHREADS_GATHER : NTHREADS, smem, st>>>(tk, tv, p);
+    };
+    if (gather) {
+      if (f32) launch(decode_split_kernel<float, true>, Lay<true>::ALLOC);
+      else launch(decode_split_kernel<__nv_bfloat16, true>, Lay<true>::ALLOC);
     } else {
-      static bool done = false;
-      if (!done) { cudaFuncSetAttribute(decode_split_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM_ALLOC); done = true; }
-      decode_split_kernel<__nv_bfloat16><<<grid, NTHREADS, SM_ALLOC, st>>>(tk, tv, p);
+      if (f32) launch(decode_split_kernel<float, false>, Lay<false>::ALLOC);
+      else launch(decode_split_kernel<__nv_bfloat16, false>, Lay<false>::ALLOC);
     }
   }
   cudaError_t e = cudaGetLastError();
