@@ -777,6 +777,8 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
 
   CUtensorMap tq, tks, tvs, tkr, tvr;
   const uint64_t self_total = (uint64_t)G * (uint64_t)a.self_rows;
+  // TMA coordinates are 32-bit row indices
+  if (self_total + TILE_N > 0x7fffffffull || (uint64_t)a.route_rows + TILE_N > 0x7fffffffull) return cudaErrorInvalidValue;
   if (!map_q(&tq, a.q, (uint64_t)a.total, Hq, s) || !map_rows(&tks, a.k_self, self_total) ||
       !map_rows(&tvs, a.v_self, self_total))
     return cudaErrorInvalidValue;

@@ -504,6 +504,7 @@ cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, 
   const int G = ctx->desc.n_kv_heads, Hq = ctx->desc.n_q_heads, s = Hq / G;
   const int ns = rc_decode_n_splits(ctx, a.batch, a.max_res_pages, a.max_hist_pages);
   const int64_t units = (int64_t)a.batch * G * ns;
+  if ((uint64_t)a.n_pages * PT > 0x7fffffffull) return cudaErrorInvalidValue;   // TMA coordinates are 32-bit row indices
   CUtensorMap tk, tv;
   if (!map_pages(&tk, a.k_pages, (uint64_t)a.n_pages) || !map_pages(&tv, a.v_pages, (uint64_t)a.n_pages))
     return cudaErrorInvalidValue;
