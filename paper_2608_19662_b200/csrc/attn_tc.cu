@@ -7,12 +7,15 @@
 // causal granularity is 128 / s tokens.  The two tiles of a CTA are consecutive
 // and share each K/V tile, read once from L2/HBM by TMA.
 //
-//   warps 0-3  softmax of tile A      warps 4-7  softmax of tile B
-//   warp  8    TMA producer           warp  9    tcgen05.mma issuer (+ TMEM alloc)
-//   warp  10   scheduler: draws work items from a global counter and publishes
-//              them through a two-slot ring in shared memory
-//   warp  11   idle (completes the third warpgroup: setmaxnreg moves registers
-//              from it to the two softmax warpgroups, 128 scores per thread)
+//   warps 0-3    softmax of tile A    warps 4-7  softmax of tile B
+//   warp  8      TMA producer         warp  9    tcgen05.mma issuer (+ TMEM alloc)
+//   warp  10     scheduler: draws work items from a global counter and publishes
+//                them through a two-slot ring in shared memory
+//   warp  11     idle (completes the third warpgroup)
+//   warps 12-15  epilogue: O of a finished tile goes from tensor memory to HBM
+//                while the softmax warps already rotate the next item's Q
+// setmaxnreg moves registers from warps 8-15 to the two softmax warpgroups,
+// which hold 128 scores per thread.
 //
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
 // S = Q K^T (both operands in 128B-swizzled shared memory, K-major); the softmax
@@ -38,8 +41,8 @@ constexpr int TILE_N = 128;
 constexpr int NSTAGE = 2;
 constexpr int BOX_BYTES = 16384;   // [128 rows][64 bf16], 128-byte swizzle
 constexpr int TILE_BYTES = 32768;  // two boxes: head_dim halves
-constexpr int NTHREADS = 384;
-constexpr int REGS_SOFTMAX = 224, REGS_AUX = 56;   // 256*224 + 128*56 = 384*168
+constexpr int NTHREADS = 512;
+constexpr int REGS_SOFTMAX = 224, REGS_AUX = 32, REGS_EPI = 32;   // 256*224 + 128*(32 + 32) = 65536
 
 constexpr int SM_Q = 0;                              // 2 query tiles
 constexpr int SM_K = SM_Q + 2 * TILE_BYTES;          // NSTAGE key tiles
@@ -49,12 +52,14 @@ constexpr int SM_ROT = SM_V + NSTAGE * TILE_BYTES;   // cos | sin of the item's 
 constexpr int SM_BAR = SM_ROT + 2 * ROT_BYTES;       // mbarriers
 constexpr int SM_MISC = SM_BAR + 32 * 8;             // tmem base, abort flag
 constexpr int SM_ITEM = SM_MISC + 64;                // two published work items
-constexpr int SM_TOTAL = SM_ITEM + 2 * 64;
+constexpr int SM_INVL = SM_ITEM + 2 * 64;            // 1 / row sum of each query tile's rows, for the epilogue warps
+constexpr int SM_TOTAL = SM_INVL + 2 * 128 * 4;
 constexpr int SM_ALLOC = SM_TOTAL + 1024;            // slack for 1024-byte alignment
 
-enum { B_QFULL = 0, B_QREADY, B_QEMPTY, B_KFULL, B_KEMPTY = B_KFULL + NSTAGE, B_VFULL = B_KEMPTY + NSTAGE,
+enum { B_QFULL = 0, B_QREADY, B_QEMPTY = B_QREADY + 2, B_KFULL, B_KEMPTY = B_KFULL + NSTAGE, B_VFULL = B_KEMPTY + NSTAGE,
        B_VEMPTY = B_VFULL + NSTAGE, B_SFULL = B_VEMPTY + NSTAGE, B_PREADY = B_SFULL + 2, B_ODONE = B_PREADY + 2,
-       B_IFULL = B_ODONE + 2, B_IEMPTY = B_IFULL + 2, B_COUNT = B_IEMPTY + 2 };
+       B_IFULL = B_ODONE + 2, B_IEMPTY = B_IFULL + 2, B_LREADY = B_IEMPTY + 2, B_ODRAIN = B_LREADY + 2,
+       B_COUNT = B_ODRAIN + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
@@ -134,18 +139,21 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A * B with A in shared memory (mma_ss2) or tensor memory (mma_ts2); descriptors are
-// given as (low word, high word): the high word (offsets, version, swizzle) is a constant, the low
-// word advances by adds.
-__device__ __forceinline__ void mma_ss2(uint32_t d, uint32_t alo, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-               "setp.ne.b32 p, %5, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-               ::"r"(d), "r"(alo), "r"(blo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
+// D[tmem] (+)= A * B with A in shared memory (mma_ss) or tensor memory (mma_ts); the 64-bit shared
+// memory descriptors advance by adds on their address field.
+__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
-__device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t blo, uint32_t hi, uint32_t idesc, uint32_t acc) {
-  asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tmov.b64 db, {%2, %3};\n\t"
-               "setp.ne.b32 p, %5, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-               ::"r"(d), "r"(a), "r"(blo), "r"(hi), "r"(idesc), "r"(acc) : "memory");
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d), "r"(a), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+// one lane of a fully converged warp, chosen by the hardware
+__device__ __forceinline__ bool elect_one() {
+  uint32_t e;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(e));
+  return e != 0;
 }
 
 #define RC_R32(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
@@ -168,6 +176,17 @@ __device__ __forceinline__ void mma_ts2(uint32_t d, uint32_t a, uint32_t blo, ui
 #define TMEM_ST32(taddr, r, o) \
   asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], " RC_LIST32_IN ";" ::"r"(taddr), RC_W32(r, o) : "memory")
 
+#define TMEM_LD16(taddr, r) \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), \
+                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) : "r"(taddr) : "memory")
+
+// one 32-byte store (the address is 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e, uint32_t f,
+                                             uint32_t g, uint32_t h) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(e),
+               "r"(f), "r"(g), "r"(h) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -319,7 +338,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     mbar_init(bar(B_QFULL), 1);
-    mbar_init(bar(B_QREADY), 256);
+    mbar_init(bar(B_QREADY + 0), 128); mbar_init(bar(B_QREADY + 1), 128);
     mbar_init(bar(B_QEMPTY), 1);
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(bar(B_KFULL + i), 1); mbar_init(bar(B_KEMPTY + i), 1);
@@ -327,7 +346,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1); mbar_init(bar(B_PREADY + x), 128); mbar_init(bar(B_ODONE + x), 1);
-      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 258);   // producer + MMA + 256 softmax threads
+      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 386);   // producer + MMA + 256 softmax + 128 epilogue threads
+      mbar_init(bar(B_LREADY + x), 128); mbar_init(bar(B_ODRAIN + x), 128);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -358,7 +378,71 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     if (release) mbar_arrive(bar(B_IEMPTY + sl));
   };
 
-  if (warp >= 8) {
+  if (warp >= 12) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_EPI));
+    // ===================== epilogue warps =====================
+    // O of a finished query tile leaves tensor memory here, so that the softmax warps can go
+    // straight to the next item's Q.  Warp 12 + q reads lanes 32 q .. 32 q + 31.
+    const int row = threadIdx.x & 127;
+    const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3)) << 16);
+    const float* inv_l = reinterpret_cast<const float*>(sm_gen + SM_INVL);
+    Item it, nx;
+    uint32_t done[2] = {0, 0};
+    fetch_item(0, it, true);
+    for (uint32_t item_n = 0; it.n_tiles > 0; ++item_n) {
+      fetch_item(item_n + 1, nx, true);
+      // The stores below and the rotation of the next item's Q go through the same load/store
+      // path, and only the rotation is urgent: let it finish first.  (O is not needed back before
+      // the next item's first P V, a whole softmax later.)
+      if (nx.n_tiles > 0) {
+        mbar_wait(bar(B_QREADY + 0), (item_n + 1u) & 1u, abort_flag, p.status);
+        mbar_wait(bar(B_QREADY + 1), (item_n + 1u) & 1u, abort_flag, p.status);
+      }
+      for (int x = 0; x < 2; ++x) {
+        if (x == 1 && !it.b_valid) continue;
+        mbar_wait(bar(B_LREADY + x), done[x] & 1u, abort_flag, p.status);
+        mbar_wait(bar(B_ODONE + x), done[x] & 1u, abort_flag, p.status);
+        ++done[x];
+        tc_fence_after();
+        const float inv = inv_l[x * 128 + row];
+        const int t_row = it.tok0 + x * TQ + row / s;
+        const bool row_valid = t_row < it.L;
+        TO* orow = reinterpret_cast<TO*>(p.out) + ((int64_t)(it.seq0 + t_row) * p.Hq + it.g * s + row % s) * D;
+        const uint32_t t_o = tmem + lane_addr + COL_O + 128 * x;
+#pragma unroll 1
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t orr[16];
+          TMEM_LD16(t_o + 16 * ch, orr);
+          tmem_wait_ld();
+          if (row_valid) {
+            if constexpr (sizeof(TO) == 4) {
+#pragma unroll
+              for (int c = 0; c < 16; c += 8)
+                st_global_v8(reinterpret_cast<float*>(orow) + 16 * ch + c,
+                             __float_as_uint(__uint_as_float(orr[c]) * inv), __float_as_uint(__uint_as_float(orr[c + 1]) * inv),
+                             __float_as_uint(__uint_as_float(orr[c + 2]) * inv), __float_as_uint(__uint_as_float(orr[c + 3]) * inv),
+                             __float_as_uint(__uint_as_float(orr[c + 4]) * inv), __float_as_uint(__uint_as_float(orr[c + 5]) * inv),
+                             __float_as_uint(__uint_as_float(orr[c + 6]) * inv), __float_as_uint(__uint_as_float(orr[c + 7]) * inv));
+            } else {
+              st_global_v8(reinterpret_cast<__nv_bfloat16*>(orow) + 16 * ch,
+                           pack2(__uint_as_float(orr[0]) * inv, __uint_as_float(orr[1]) * inv),
+                           pack2(__uint_as_float(orr[2]) * inv, __uint_as_float(orr[3]) * inv),
+                           pack2(__uint_as_float(orr[4]) * inv, __uint_as_float(orr[5]) * inv),
+                           pack2(__uint_as_float(orr[6]) * inv, __uint_as_float(orr[7]) * inv),
+                           pack2(__uint_as_float(orr[8]) * inv, __uint_as_float(orr[9]) * inv),
+                           pack2(__uint_as_float(orr[10]) * inv, __uint_as_float(orr[11]) * inv),
+                           pack2(__uint_as_float(orr[12]) * inv, __uint_as_float(orr[13]) * inv),
+                           pack2(__uint_as_float(orr[14]) * inv, __uint_as_float(orr[15]) * inv));
+            }
+          }
+        }
+        // the next item's first P V overwrites O, its softmax overwrites 1 / l: both wait for this
+        tc_fence_before();
+        mbar_arrive(bar(B_ODRAIN + x));
+      }
+      it = nx;
+    }
+  } else if (warp >= 8) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_AUX));
   if (warp == 10) {
     // ===================== scheduler =====================
@@ -433,28 +517,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   } else if (warp == 9) {
     // ===================== MMA issuer =====================
     // descriptor words: low = (address >> 4) | (LBO >> 4) << 16, high = (SBO >> 4) | version | swizzle
-    const uint64_t d_k = smem_desc(0, 16, 1024), d_v = smem_desc(0, BOX_BYTES, 1024);
-    const uint32_t hi_k = (uint32_t)(d_k >> 32), hi_v = (uint32_t)(d_v >> 32);
-    const uint32_t lo_q = (uint32_t)d_k + ((sm + SM_Q) >> 4), lo_k = (uint32_t)d_k + ((sm + SM_K) >> 4);
-    const uint32_t lo_v = (uint32_t)d_v + ((sm + SM_V) >> 4);
+    // The issuing lane is elected once: every MMA and every commit comes from that one thread
+    // (a commit tracks the MMAs of the thread that executes it).
+    const bool issuer = elect_one();
+    const uint64_t d_q = smem_desc(0, 16, 1024) + ((sm + SM_Q) >> 4), d_k = smem_desc(0, 16, 1024) + ((sm + SM_K) >> 4);
+    const uint64_t d_v = smem_desc(0, BOX_BYTES, 1024) + ((sm + SM_V) >> 4);
     auto issue_qk = [&](int x, int st) {
-      const uint32_t qa = lo_q + x * (TILE_BYTES >> 4), ka = lo_k + st * (TILE_BYTES >> 4);
+      const uint64_t qa = d_q + x * (TILE_BYTES >> 4), ka = d_k + st * (TILE_BYTES >> 4);
       const uint32_t dst = tmem + COL_S + 128 * x;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint32_t off = ((j >> 2) * BOX_BYTES + (j & 3) * 32) >> 4;
-        mma_ss2(dst, qa + off, ka + off, hi_k, IDESC_QK, j > 0);
+        mma_ss(dst, qa + off, ka + off, IDESC_QK, j > 0);
       }
     };
     auto issue_pv = [&](int x, int st, int ksteps, bool first) {
-      const uint32_t va = lo_v + st * (TILE_BYTES >> 4);
+      const uint64_t va = d_v + st * (TILE_BYTES >> 4);
       const uint32_t dst = tmem + COL_O + 128 * x, src = tmem + COL_S + 128 * x;
 #pragma unroll 8
       for (int j = 0; j < ksteps; ++j)
-        mma_ts2(dst, src + 8 * j, va + j * (2048 >> 4), hi_v, IDESC_PV, (!first || j > 0) ? 1u : 0u);
+        mma_ts(dst, src + 8 * j, va + j * (2048 >> 4), IDESC_PV, (!first || j > 0) ? 1u : 0u);
     };
     Item it;
     uint32_t kv_n = 0, cnt[2] = {0, 0};   // K/V tiles, tiles per query tile so far
+    uint32_t items_x[2] = {0, 0};         // items each query tile has taken part in
     for (uint32_t item_n = 0;; ++item_n) {
       fetch_item(item_n, it, false);
       __syncwarp();
@@ -462,14 +548,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       if (it.n_tiles < 0) break;
       const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, L = it.H + it.L, kv_end = it.kv_end;
       const bool b_valid = it.b_valid != 0;
-      mbar_wait(bar(B_QREADY), item_n & 1u, abort_flag, p.status);
+      // each query tile starts as soon as its own half of Q has been rotated
+      mbar_wait(bar(B_QREADY + 0), item_n & 1u, abort_flag, p.status);
       mbar_wait(bar(B_KFULL + kv_n % NSTAGE), (kv_n / NSTAGE) & 1u, abort_flag, p.status);
       tc_fence_after();
-      if (lane == 0) {
-        const int st0 = kv_n % NSTAGE;
-        issue_qk(0, st0); tc_commit(bar(B_SFULL + 0));
+      const int st0 = kv_n % NSTAGE;
+      if (issuer) { issue_qk(0, st0); tc_commit(bar(B_SFULL + 0)); }
+      // (waited for even when the second tile is empty: its warps still rewrite that half of Q,
+      // and the Q-empty commit below lets the next load overwrite it)
+      mbar_wait(bar(B_QREADY + 1), item_n & 1u, abort_flag, p.status);
+      tc_fence_after();
+      if (issuer) {
         if (b_valid) { issue_qk(1, st0); tc_commit(bar(B_SFULL + 1)); }
-        tc_commit(bar(B_KEMPTY + st0));
         if (n_tiles == 1) tc_commit(bar(B_QEMPTY));
       }
       __syncwarp();
@@ -496,32 +586,34 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const int st1 = (n + 1) % NSTAGE;
         const uint32_t ph1 = ((n + 1) / NSTAGE) & 1u;
         const bool more = i + 1 < n_tiles;
-        mbar_wait(bar(B_PREADY + 0), cnt[0] & 1u, abort_flag, p.status);
+        mbar_wait(bar(B_PREADY + 0), cnt[0]++ & 1u, abort_flag, p.status);
+        if (i == 0 && items_x[0] > 0) mbar_wait(bar(B_ODRAIN + 0), (items_x[0] - 1u) & 1u, abort_flag, p.status);
         tc_fence_after();
-        if (lane == 0) { issue_pv(0, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 0)); }
-        ++cnt[0];
+        if (issuer) { issue_pv(0, st, ksteps, i == 0); if (!more) tc_commit(bar(B_ODONE + 0)); }
         if (more) {
           mbar_wait(bar(B_KFULL + st1), ph1, abort_flag, p.status);
           tc_fence_after();
-          if (lane == 0) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
+          if (issuer) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
         }
         if (b_valid) {
-          mbar_wait(bar(B_PREADY + 1), cnt[1] & 1u, abort_flag, p.status);
+          mbar_wait(bar(B_PREADY + 1), cnt[1]++ & 1u, abort_flag, p.status);
+          if (i == 0 && items_x[1] > 0) mbar_wait(bar(B_ODRAIN + 1), (items_x[1] - 1u) & 1u, abort_flag, p.status);
           tc_fence_after();
-          if (lane == 0) { issue_pv(1, st, ksteps, i == 0); tc_commit(bar(B_ODONE + 1)); }
-          ++cnt[1];
+          if (issuer) { issue_pv(1, st, ksteps, i == 0); if (!more) tc_commit(bar(B_ODONE + 1)); }
         }
-        if (lane == 0) {
-          tc_commit(bar(B_VEMPTY + st));
+        if (issuer) {
           if (more) {
             if (b_valid) { issue_qk(1, st1); tc_commit(bar(B_SFULL + 1)); }
-            tc_commit(bar(B_KEMPTY + st1));
             if (i + 2 == n_tiles) tc_commit(bar(B_QEMPTY));   // the item's last S has been issued
+          } else {
+            tc_commit(bar(B_VEMPTY + st));                    // the item's last V tile (earlier ones: see the softmax side)
           }
         }
         __syncwarp();
       }
       kv_n += (uint32_t)n_tiles;
+      ++items_x[0];
+      if (b_valid) ++items_x[1];
     }
   }
   } else {
@@ -534,50 +626,59 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const uint32_t t_o = tmem + lane_addr + COL_O + 128 * x;
     const float c2 = p.scale_log2;
     uint32_t item_n = 0, cnt = 0;                  // items seen; tiles this query tile has gone through
+    uint32_t kv_n = 0, done_n = 0;                 // K/V tiles of all items so far; items this query tile took part in
 
-    // Rotates this thread's row of the freshly loaded Q tile in shared memory
-    // (swizzled 16-byte chunks; element i pairs with i + 64 in the other box).
+    // Rotates this query tile of the freshly loaded Q in shared memory (swizzled 16-byte chunks;
+    // element i pairs with i + 64 in the other box).  A thread takes one (token, chunk) pair at a
+    // time and goes through the token's s heads, so that cos / sin are read once per token, not
+    // once per row; the 8 lanes of a token cover whole 128-byte rows of Q.
     auto rotate_q = [&](const Item& it, uint32_t n_item) {
       mbar_wait(bar(B_QFULL), n_item & 1u, abort_flag, p.status);
-      const int t_eff = min(it.tok0 + x * TQ + row / s, it.L - 1);
-      const int pos = it.pos0 + t_eff;
-      if (pos < 0 || pos >= p.max_pos) rc_set_status(p.status, RECACHE_DEV_BAD_POS);
-      const float4 *cp, *sp;
-      if (ROT_SMEM) {   // staged by the producer: row = token index inside the tile pair
-        const int ri = min(max(t_eff - it.tok0, 0), 2 * TQ - 1);
-        cp = reinterpret_cast<const float4*>(sm_gen + SM_ROT + ri * 256);
-        sp = reinterpret_cast<const float4*>(sm_gen + SM_ROT + ROT_BYTES + ri * 256);
-      } else {
-        const int pc = min(max(pos, 0), p.max_pos - 1);
-        cp = reinterpret_cast<const float4*>(p.cos_tab + (int64_t)pc * 64);
-        sp = reinterpret_cast<const float4*>(p.sin_tab + (int64_t)pc * 64);
-      }
-      uint8_t* qb = sm_gen + SM_Q + x * TILE_BYTES + row * 128;
-#pragma unroll
-      for (int cc = 0; cc < 8; ++cc) {
-        // threads of a warp read 8 different cos/sin rows 256 bytes apart: start each row at another chunk
-        const int c = (cc + row / s) & 7;
-        const int off = ((c ^ (row & 7)) << 4);
-        const uint4 ulo = *reinterpret_cast<uint4*>(qb + off), uhi = *reinterpret_cast<uint4*>(qb + BOX_BYTES + off);
-        const float4 c0 = cp[2 * c], c1 = cp[2 * c + 1], s0 = sp[2 * c], s1 = sp[2 * c + 1];
+      uint8_t* qt = sm_gen + SM_Q + x * TILE_BYTES;
+      for (int u = row; u < TQ * 8; u += 128) {
+        const int tok = u >> 3, c = u & 7;
+        const int t_eff = min(it.tok0 + x * TQ + tok, it.L - 1);
+        const int pos = it.pos0 + t_eff;
+        if (pos < 0 || pos >= p.max_pos) rc_set_status(p.status, RECACHE_DEV_BAD_POS);
+        const float *cp, *sp;
+        if (ROT_SMEM) {   // staged by the producer: row = token index inside the tile pair
+          const int ri = min(max(t_eff - it.tok0, 0), 2 * TQ - 1);
+          cp = reinterpret_cast<const float*>(sm_gen + SM_ROT + ri * 256) + c * 8;
+          sp = reinterpret_cast<const float*>(sm_gen + SM_ROT + ROT_BYTES + ri * 256) + c * 8;
+        } else {
+          const int pc = min(max(pos, 0), p.max_pos - 1);
+          cp = p.cos_tab + (int64_t)pc * 64 + c * 8;
+          sp = p.sin_tab + (int64_t)pc * 64 + c * 8;
+        }
+        // lanes c and c + 4 would hit the same banks: they take the two halves in opposite order
+        const int first = (c & 4) ? 4 : 0;
+        const float4 ca = *reinterpret_cast<const float4*>(cp + first), cb = *reinterpret_cast<const float4*>(cp + 4 - first);
+        const float4 sa = *reinterpret_cast<const float4*>(sp + first), sb = *reinterpret_cast<const float4*>(sp + 4 - first);
+        const float4 c0 = first ? cb : ca, c1 = first ? ca : cb, s0 = first ? sb : sa, s1 = first ? sa : sb;
         const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
         const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        const uint32_t wlo[4] = {ulo.x, ulo.y, ulo.z, ulo.w}, whi[4] = {uhi.x, uhi.y, uhi.z, uhi.w};
-        uint32_t ol[4], oh[4];
+#pragma unroll 2
+        for (int h = 0; h < s; ++h) {
+          const int r = tok * s + h;
+          uint8_t* qb = qt + r * 128 + ((c ^ (r & 7)) << 4);
+          const uint4 ulo = *reinterpret_cast<uint4*>(qb), uhi = *reinterpret_cast<uint4*>(qb + BOX_BYTES);
+          const uint32_t wlo[4] = {ulo.x, ulo.y, ulo.z, ulo.w}, whi[4] = {uhi.x, uhi.y, uhi.z, uhi.w};
+          uint32_t ol[4], oh[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float l0 = __uint_as_float(wlo[i] << 16), l1 = __uint_as_float(wlo[i] & 0xffff0000u);
-          const float h0 = __uint_as_float(whi[i] << 16), h1 = __uint_as_float(whi[i] & 0xffff0000u);
-          ol[i] = pack2(__fmaf_rn(l0, cs[2 * i], -__fmul_rn(h0, sn[2 * i])),
-                        __fmaf_rn(l1, cs[2 * i + 1], -__fmul_rn(h1, sn[2 * i + 1])));
-          oh[i] = pack2(__fmaf_rn(h0, cs[2 * i], __fmul_rn(l0, sn[2 * i])),
-                        __fmaf_rn(h1, cs[2 * i + 1], __fmul_rn(l1, sn[2 * i + 1])));
+          for (int i = 0; i < 4; ++i) {
+            const float l0 = __uint_as_float(wlo[i] << 16), l1 = __uint_as_float(wlo[i] & 0xffff0000u);
+            const float h0 = __uint_as_float(whi[i] << 16), h1 = __uint_as_float(whi[i] & 0xffff0000u);
+            ol[i] = pack2(__fmaf_rn(l0, cs[2 * i], -__fmul_rn(h0, sn[2 * i])),
+                          __fmaf_rn(l1, cs[2 * i + 1], -__fmul_rn(h1, sn[2 * i + 1])));
+            oh[i] = pack2(__fmaf_rn(h0, cs[2 * i], __fmul_rn(l0, sn[2 * i])),
+                          __fmaf_rn(h1, cs[2 * i + 1], __fmul_rn(l1, sn[2 * i + 1])));
+          }
+          *reinterpret_cast<uint4*>(qb) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+          *reinterpret_cast<uint4*>(qb + BOX_BYTES) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
         }
-        *reinterpret_cast<uint4*>(qb + off) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-        *reinterpret_cast<uint4*>(qb + BOX_BYTES + off) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
       }
       fence_async_smem();
-      mbar_arrive(bar(B_QREADY));
+      mbar_arrive(bar(B_QREADY + x));
     };
 
     Item it, nx;
@@ -585,6 +686,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     if (it.n_tiles > 0) rotate_q(it, 0);
     while (it.n_tiles > 0) {
       const bool active = x == 0 || it.b_valid;
+      const bool releaser = row == 0 && x == (it.b_valid ? 1 : 0);   // the tile whose S = Q K^T is issued last
       const int t_row = it.tok0 + x * TQ + row / s;     // token (local index)
       const int t_eff = min(t_row, it.L - 1);
       const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, H = it.H;
@@ -593,6 +695,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         for (int i = 0; i < n_tiles; ++i, ++cnt) {
           mbar_wait(bar(B_SFULL + x), cnt & 1u, abort_flag, p.status);
           tc_fence_after();
+          if (releaser) {
+            // S of tile i is complete: so is every earlier MMA, i.e. the last reader of K tile i
+            // and of V tile i - 1.  Hand both stages back to the producer.
+            mbar_arrive(bar(B_KEMPTY + (kv_n + i) % NSTAGE));
+            if (i > 0) mbar_arrive(bar(B_VEMPTY + (kv_n + i - 1) % NSTAGE));
+          }
           uint32_t sr[128];
           TMEM_LD32(t_s + 0, sr, 0); TMEM_LD32(t_s + 32, sr, 32); TMEM_LD32(t_s + 64, sr, 64); TMEM_LD32(t_s + 96, sr, 96);
           tmem_wait_ld();
@@ -616,8 +724,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           if (i == 0) m_ref = m_new;                       // O is overwritten by the first P V
           else need = (m_new - m_ref) * c2 > 8.f;          // lazy: P stays below 2^8 otherwise
           if (__any_sync(0xffffffffu, need)) {
-            mbar_wait(bar(B_ODONE + x), (cnt - 1u) & 1u, abort_flag, p.status);
-            tc_fence_after();
+            // the previous P V of this tile was issued before this S, so it is complete as well
             const float f = need ? ex2((m_ref - m_new) * c2) : 1.f;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
@@ -653,41 +760,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           mbar_arrive(bar(B_PREADY + x));
         }
       }
-      // ---- next item's Q first (its load was issued a tile ago), then this item's epilogue ----
+      // ---- hand the finished tile to the epilogue warps (they wait for its last P V themselves) ----
+      if (active) {
+        if (done_n > 0) mbar_wait(bar(B_ODRAIN + x), (done_n - 1u) & 1u, abort_flag, p.status);   // 1 / l of the item before was read
+        reinterpret_cast<float*>(sm_gen + SM_INVL)[x * 128 + row] = 1.f / l_sum;
+        mbar_arrive(bar(B_LREADY + x));
+        ++done_n;
+      }
+      kv_n += (uint32_t)n_tiles;
+      // ---- next item's Q (its load was issued a tile ago) ----
       fetch_item(item_n + 1, nx, true);
       if (nx.n_tiles > 0) rotate_q(nx, item_n + 1);
-      if (active) {
-        mbar_wait(bar(B_ODONE + x), (cnt - 1u) & 1u, abort_flag, p.status);
-        tc_fence_after();
-        const float inv = 1.f / l_sum;
-        const bool row_valid = t_row < it.L;
-        TO* orow = reinterpret_cast<TO*>(p.out) + ((int64_t)(it.seq0 + t_row) * p.Hq + it.g * s + row % s) * D;
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t orr[32];
-          TMEM_LD32(t_o + 32 * ch, orr, 0);
-          tmem_wait_ld();
-          if (row_valid) {
-            if constexpr (sizeof(TO) == 4) {
-#pragma unroll
-              for (int c = 0; c < 32; c += 4)
-                *reinterpret_cast<float4*>(reinterpret_cast<float*>(orow) + 32 * ch + c) =
-                    make_float4(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv,
-                                __uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 32; c += 8)
-                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(orow) + 32 * ch + c) =
-                    make_uint4(pack2(__uint_as_float(orr[c]) * inv, __uint_as_float(orr[c + 1]) * inv),
-                               pack2(__uint_as_float(orr[c + 2]) * inv, __uint_as_float(orr[c + 3]) * inv),
-                               pack2(__uint_as_float(orr[c + 4]) * inv, __uint_as_float(orr[c + 5]) * inv),
-                               pack2(__uint_as_float(orr[c + 6]) * inv, __uint_as_float(orr[c + 7]) * inv));
-            }
-          }
-        }
-        // the next item's first P V overwrites O: order this thread's reads before its next P-ready arrive
-        tc_fence_before();
-      }
       it = nx; ++item_n;
     }
   }
