@@ -64,10 +64,13 @@ static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
 
+constexpr int SORT_MAX = 4096;                      // work items up to which the plan sorts them by weight
+
 constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long is a bug, not load
 
 struct TcParams {
-  const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter
+  const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter, header[2] = order[] is valid
+  const int32_t* order;                 // work indices, heaviest first (launches of at most SORT_MAX work items)
   const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu; const int32_t* hist;
   int n_seq, G, Hq, s;
   int prefix_len;   // > 0: every sequence sees rows g*prefix_len .. of the "route" tensors (shared prefix)
@@ -230,48 +233,6 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
-// ------------------------------------------------------------- work list --
-// Items = (sequence, tile-pair index): sequence by sequence, and inside a
-// sequence the last (heaviest) tile pair first.  With the KV group as the
-// fastest index of the flattened work list, the CTAs that run at the same time
-// share one sequence's K/V, which then stays in L2 instead of being streamed
-// from HBM once per tile pair.  One CTA; level_off[b] = first item of sequence b.
-__global__ void __launch_bounds__(1024) tile_plan_kernel(const int32_t* __restrict__ cu, int n_seq, int tok_per_cta,
-                                                         int n_levels, int32_t* __restrict__ header,
-                                                         int2* __restrict__ items, int32_t* __restrict__ level_off,
-                                                         int max_items, int32_t* status) {
-  __shared__ int chunk_sum[1024];
-  // each thread owns a contiguous chunk of sequences: local sums, scan of the chunk sums, then the items
-  const int per = (n_seq + blockDim.x - 1) / blockDim.x;
-  const int b0 = min(n_seq, (int)threadIdx.x * per), b1 = min(n_seq, b0 + per);
-  int sum = 0;
-  for (int b = b0; b < b1; ++b) {
-    const int len = cu[b + 1] - cu[b];
-    if (len < 0) rc_set_status(status, RECACHE_DEV_BAD_SEQLENS);
-    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
-    if (nt > n_levels) { rc_set_status(status, RECACHE_DEV_BAD_SEQLENS); nt = n_levels; }   // longer than the max_len given
-    sum += nt;
-  }
-  chunk_sum[threadIdx.x] = sum;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int run = 0;
-    for (int t = 0; t < (int)blockDim.x; ++t) { const int c = chunk_sum[t]; chunk_sum[t] = run; run += c; }
-    header[0] = run < max_items ? run : max_items;
-    header[1] = 0;   // dynamic work counter of the attention kernel
-  }
-  __syncthreads();
-  int k = chunk_sum[threadIdx.x];
-  for (int b = b0; b < b1; ++b) {
-    const int len = cu[b + 1] - cu[b];
-    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
-    if (nt > n_levels) nt = n_levels;
-    level_off[b] = k;
-    for (int l = nt - 1; l >= 0; --l, ++k)
-      if (k < max_items) items[k] = make_int2(b, l);
-  }
-}
-
 // One work item as published by the scheduler warp (16 ints in shared memory).
 struct Item {
   int n_tiles;      // -1: no more work
@@ -308,10 +269,109 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
   return ok;
 }
 
+// ------------------------------------------------------------- work list --
+// Items = (sequence, tile-pair index): sequence by sequence, and inside a
+// sequence the last (heaviest) tile pair first.  With the KV group as the
+// fastest index of the flattened work list, the CTAs that run at the same time
+// share one sequence's K/V, which then stays in L2 instead of being streamed
+// from HBM once per tile pair.  One CTA; level_off[b] = first item of sequence b.
+__global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int tok_per_cta, int n_levels,
+                                                         int2* __restrict__ items, int32_t* __restrict__ level_off,
+                                                         int32_t* __restrict__ order, int max_items) {
+  __shared__ int warp_sum[32];
+  __shared__ int hist[1025];
+  const int n_seq = p.n_seq;
+  const int32_t* cu = p.cu;
+  // each thread owns a contiguous chunk of sequences: local sums, block scan of the chunk sums, then the items
+  const int per = (n_seq + blockDim.x - 1) / blockDim.x;
+  const int b0 = min(n_seq, (int)threadIdx.x * per), b1 = min(n_seq, b0 + per);
+  int sum = 0;
+  for (int b = b0; b < b1; ++b) {
+    const int len = cu[b + 1] - cu[b];
+    if (len < 0) rc_set_status(p.status, RECACHE_DEV_BAD_SEQLENS);
+    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+    if (nt > n_levels) { rc_set_status(p.status, RECACHE_DEV_BAD_SEQLENS); nt = n_levels; }   // longer than the max_len given
+    sum += nt;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = sum;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += v;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sum[lane], wi = w;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += v;
+    }
+    warp_sum[lane] = wi - w;   // exclusive
+    if (lane == 31) {
+      p.header[0] = wi < max_items ? wi : max_items;
+      p.header[1] = 0;         // dynamic work counter of the attention kernel
+    }
+  }
+  __syncthreads();
+  int k = warp_sum[warp] + incl - sum;
+  for (int b = b0; b < b1; ++b) {
+    const int len = cu[b + 1] - cu[b];
+    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+    if (nt > n_levels) nt = n_levels;
+    level_off[b] = k;
+    for (int l = nt - 1; l >= 0; --l, ++k)
+      if (k < max_items) items[k] = make_int2(b, l);
+  }
+  // Few work items (a prefill of a handful of requests): one CTA gets one or two of them, so their
+  // order decides the tail.  Sort them by weight (K/V tiles), heaviest first, with a counting sort.
+  __syncthreads();
+  const int n_work = p.header[0] * p.G;
+  const bool sorted = n_work <= SORT_MAX;
+  if (threadIdx.x == 0) p.header[2] = sorted ? 1 : 0;
+  if (!sorted) return;
+  for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  int bin[SORT_MAX / 1024];
+#pragma unroll
+  for (int j = 0; j < SORT_MAX / 1024; ++j) {
+    const int w = threadIdx.x + j * 1024;
+    bin[j] = -1;
+    if (w < n_work) {
+      Item it;
+      const bool ok = load_item(p, w, it);
+      bin[j] = 1024 - (ok ? min(it.n_tiles, 1024) : 0);   // heaviest first
+      atomicAdd(&hist[bin[j]], 1);
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {   // exclusive scan of the 1025 bins
+    int carry = 0;
+    for (int c0 = 0; c0 < 1025; c0 += 32) {
+      const int v = c0 + lane < 1025 ? hist[c0 + lane] : 0;
+      int vi = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, vi, off);
+        if (lane >= off) vi += u;
+      }
+      if (c0 + lane < 1025) hist[c0 + lane] = carry + vi - v;
+      carry += __shfl_sync(0xffffffffu, vi, 31);
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < SORT_MAX / 1024; ++j)
+    if (bin[j] >= 0) order[atomicAdd(&hist[bin[j]], 1)] = threadIdx.x + j * 1024;
+}
+
 // ---------------------------------------------------------------- kernel --
 // Persistent: a scheduler warp draws work indices from a global counter (the
-// list is heavy-first inside each sequence, so the tail of the launch is made of
-// light items) and publishes items through a two-slot ring in shared memory.
+// list is heavy-first inside each sequence, or heavy-first overall when the plan
+// sorted it, so the tail of the launch is made of light items) and publishes
+// items through a two-slot ring in shared memory.
 // The next item's Q load, Q rotation and first K/V tiles overlap the current
 // item's last tiles and its epilogue.  Barrier phases run on across items.
 template <typename TO, bool ROT_SMEM>
@@ -456,7 +516,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           const int w = first ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(p.header + 1, 1);
           first = false;
           if (w >= total || *abort_flag) { it.n_tiles = -1; break; }
-          if (load_item(p, w, it)) break;
+          if (load_item(p, p.header[2] ? p.order[w] : w, it)) break;
         }
         volatile int* r = item_ring + sl * IT_WORDS;
         r[IT_NTILES] = it.n_tiles;
@@ -845,7 +905,7 @@ static int tc_levels(const recache_ctx* ctx, int max_len) {
 }
 
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len) {
-  return 256 + align256(tc_max_items(ctx, n_seq, total) * 8) + align256((int64_t)(n_seq + 1) * 4);
+  return 256 + align256(tc_max_items(ctx, n_seq, total) * 8) + align256((int64_t)(n_seq + 1) * 4) + align256(SORT_MAX * 4);
 }
 
 cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaStream_t st) {
@@ -857,6 +917,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   int32_t* header = (int32_t*)ws;
   int2* items = (int2*)(ws + 256);
   int32_t* level_off = (int32_t*)(ws + 256 + align256(max_items * 8));
+  int32_t* order = (int32_t*)(ws + 256 + align256(max_items * 8) + align256((int64_t)(a.n_seq + 1) * 4));
 
   CUtensorMap tq, tks, tvs, tkr, tvr;
   const uint64_t self_total = (uint64_t)G * (uint64_t)a.self_rows;
@@ -870,11 +931,6 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
       !map_rows(&tvr, has_route ? a.v_route : a.v_self, has_route ? (uint64_t)a.route_rows : self_total))
     return cudaErrorInvalidValue;
 
-  {
-    RcLaunchScope scope(ctx, RC_K_TILE_PLAN, st);
-    tile_plan_kernel<<<1, 1024, 0, st>>>(a.cu, a.n_seq, tc_tok_per_cta(ctx), n_levels, header, items, level_off,
-                                         (int)max_items, ctx->status);
-  }
   TcParams p;
   p.items = items; p.header = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
   p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.out = a.o;
@@ -883,6 +939,11 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)ctx->desc.head_dim));
   p.status = ctx->status;
+  p.order = order;
+  {
+    RcLaunchScope scope(ctx, RC_K_TILE_PLAN, st);
+    tile_plan_kernel<<<1, 1024, 0, st>>>(p, tc_tok_per_cta(ctx), n_levels, items, level_off, order, (int)max_items);
+  }
   const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
   const unsigned grid = (unsigned)(max_items * G < sms ? max_items * G : sms);
   RcLaunchScope scope(ctx, a.route_cu ? RC_K_PREFILL_ATTN : RC_K_ENCODE_ATTN, st);
