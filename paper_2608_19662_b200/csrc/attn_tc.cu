@@ -59,7 +59,7 @@ constexpr int SM_ALLOC = SM_TOTAL + 1024;            // slack for 1024-byte alig
 enum { B_QFULL = 0, B_QREADY, B_QEMPTY = B_QREADY + 2, B_KFULL, B_KEMPTY = B_KFULL + NSTAGE, B_VFULL = B_KEMPTY + NSTAGE,
        B_VEMPTY = B_VFULL + NSTAGE, B_SFULL = B_VEMPTY + NSTAGE, B_PREADY = B_SFULL + 2, B_ODONE = B_PREADY + 2,
        B_IFULL = B_ODONE + 2, B_IEMPTY = B_IFULL + 2, B_LREADY = B_IEMPTY + 2, B_ODRAIN = B_LREADY + 2,
-       B_COUNT = B_ODRAIN + 2 };
+       B_PHALF = B_ODRAIN + 2, B_COUNT = B_PHALF + 2 };
 static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1); mbar_init(bar(B_PREADY + x), 128); mbar_init(bar(B_ODONE + x), 1);
       mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 386);   // producer + MMA + 256 softmax + 128 epilogue threads
-      mbar_init(bar(B_LREADY + x), 128); mbar_init(bar(B_ODRAIN + x), 128);
+      mbar_init(bar(B_LREADY + x), 128); mbar_init(bar(B_ODRAIN + x), 128); mbar_init(bar(B_PHALF + x), 128);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -591,11 +591,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         mma_ss(dst, qa + off, ka + off, IDESC_QK, j > 0);
       }
     };
-    auto issue_pv = [&](int x, int st, int ksteps, bool first) {
+    auto issue_pv = [&](int x, int st, int k0, int ksteps, bool first) {
       const uint64_t va = d_v + st * (TILE_BYTES >> 4);
       const uint32_t dst = tmem + COL_O + 128 * x, src = tmem + COL_S + 128 * x;
-#pragma unroll 8
-      for (int j = 0; j < ksteps; ++j)
+#pragma unroll 4
+      for (int j = k0; j < ksteps; ++j)
         mma_ts(dst, src + 8 * j, va + j * (2048 >> 4), IDESC_PV, (!first || j > 0) ? 1u : 0u);
     };
     Item it;
@@ -646,20 +646,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const int st1 = (n + 1) % NSTAGE;
         const uint32_t ph1 = ((n + 1) / NSTAGE) & 1u;
         const bool more = i + 1 < n_tiles;
-        mbar_wait(bar(B_PREADY + 0), cnt[0]++ & 1u, abort_flag, p.status);
+        // P of keys 0..63 arrives first: half of P V runs while the softmax finishes the other half
+        mbar_wait(bar(B_PHALF + 0), cnt[0] & 1u, abort_flag, p.status);
         if (i == 0 && items_x[0] > 0) mbar_wait(bar(B_ODRAIN + 0), (items_x[0] - 1u) & 1u, abort_flag, p.status);
         tc_fence_after();
-        if (issuer) { issue_pv(0, st, ksteps, i == 0); if (!more) tc_commit(bar(B_ODONE + 0)); }
+        if (issuer) issue_pv(0, st, 0, min(ksteps, 4), i == 0);
+        mbar_wait(bar(B_PREADY + 0), cnt[0]++ & 1u, abort_flag, p.status);
+        tc_fence_after();
+        if (issuer) { issue_pv(0, st, 4, ksteps, false); if (!more) tc_commit(bar(B_ODONE + 0)); }
         if (more) {
           mbar_wait(bar(B_KFULL + st1), ph1, abort_flag, p.status);
           tc_fence_after();
           if (issuer) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
         }
         if (b_valid) {
-          mbar_wait(bar(B_PREADY + 1), cnt[1]++ & 1u, abort_flag, p.status);
+          mbar_wait(bar(B_PHALF + 1), cnt[1] & 1u, abort_flag, p.status);
           if (i == 0 && items_x[1] > 0) mbar_wait(bar(B_ODRAIN + 1), (items_x[1] - 1u) & 1u, abort_flag, p.status);
           tc_fence_after();
-          if (issuer) { issue_pv(1, st, ksteps, i == 0); if (!more) tc_commit(bar(B_ODONE + 1)); }
+          if (issuer) issue_pv(1, st, 0, min(ksteps, 4), i == 0);
+          mbar_wait(bar(B_PREADY + 1), cnt[1]++ & 1u, abort_flag, p.status);
+          tc_fence_after();
+          if (issuer) { issue_pv(1, st, 4, ksteps, false); if (!more) tc_commit(bar(B_ODONE + 1)); }
         }
         if (issuer) {
           if (more) {
@@ -811,7 +818,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             add2(acc[2], acc[3], p2, p3);
             pr[c] = pack2(p0, p1);
             pr[c + 1] = pack2(p2, p3);
-            if (c == 30) TMEM_ST32(t_s + 0, pr, 0);        // first half of P goes out while the second is computed
+            if (c == 30) {   // first half of P goes out, and into P V, while the second is computed
+              TMEM_ST32(t_s + 0, pr, 0);
+              tmem_wait_st();
+              tc_fence_before();
+              mbar_arrive(bar(B_PHALF + x));
+            }
           }
           l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
           TMEM_ST32(t_s + 32, pr, 32);
