@@ -64,7 +64,7 @@ static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
 
-constexpr int SORT_MAX = 4096;                      // work items up to which the plan sorts them by weight
+constexpr int SORT_MAX = 1024;                      // work items up to which the plan sorts them by weight
 
 constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long is a bug, not load
 
