@@ -64,7 +64,7 @@ static_assert(B_COUNT <= 32, "barrier area");
 
 constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
 
-constexpr int SORT_MAX = 1024;                      // work items up to which the plan sorts them by weight
+constexpr int SORT_MAX = 4096;                      // work items up to which the plan sorts a prefill by weight (encode: a quarter)
 
 constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long is a bug, not load
 
@@ -329,7 +329,9 @@ __global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int t
   // order decides the tail.  Sort them by weight (K/V tiles), heaviest first, with a counting sort.
   __syncthreads();
   const int n_work = p.header[0] * p.G;
-  const bool sorted = n_work <= SORT_MAX;
+  // (an encode launch shares K/V between the items of a sequence only: beyond a thousand items the
+  // sequence-major order, which keeps a sequence's K/V in L2, is worth more than the balance)
+  const bool sorted = n_work <= (p.route_cu ? SORT_MAX : SORT_MAX / 4);
   if (threadIdx.x == 0) p.header[2] = sorted ? 1 : 0;
   if (!sorted) return;
   for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
