@@ -258,6 +258,28 @@ RECACHE_API recache_status recache_attend_prefill_history(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
+ * Routed prefill without materialising the route rows (zero-copy; the paper's
+ * request-local KV materialisation replaced by an index list): route b*G+g is
+ * rows route_idx[route_cu[r] .. route_cu[r+1]) of group g of the resource cache
+ * k_cache / v_cache [G][pool_tokens][d] - what recache_compact_routes writes when
+ * called with k_out = v_out = NULL in packed mode.  route_rows = entries of
+ * route_idx.  Same mask, same softmax, same tiles as recache_attend_prefill on
+ * the packed rows: the results are bit-identical to it.
+ * bf16 contexts with head_dim 128 and 2, 4 or 8 query heads per KV head only
+ * (RECACHE_EUNSUPPORTED otherwise).  An index outside [0, pool_tokens) sets the
+ * device status (bad slot) and its row is read as zeros.
+ */
+RECACHE_API recache_status recache_attend_prefill_gather(recache_ctx* ctx,
+    const void* q, const void* k_conv, const void* v_conv,
+    const int32_t* cu_q, const int32_t* q_pos0,
+    int32_t n_requests, int32_t total_q, int32_t max_q,
+    const void* k_cache, const void* v_cache, int64_t pool_tokens,
+    const int32_t* route_idx, const int32_t* route_cu, int64_t route_rows,
+    void* k_conv_out, void* v_conv_out,
+    void* out_o, int32_t out_dtype,
+    void* workspace, int64_t workspace_bytes, void* stream);
+
+/*
  * Routed decode (paper: the same mask "during decoding"; the Attn. latency of
  * the efficiency study).  One query token per sequence at position q_pos[b].
  * Item it = b * G + g reads res_len[it] rows through res_page_table[it][*] and

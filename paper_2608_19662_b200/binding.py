@@ -51,6 +51,8 @@ SIGNATURES = {
                                          _I64, _P, _P, _P, _I32, _P, _I64, _I64, _P, _I64, _P]),
     "recache_attend_prefill": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
                                          _P, _I32, _P, _I64, _P]),
+    "recache_attend_prefill_gather": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _I64, _P, _P, _I64,
+                                                _P, _P, _P, _I32, _P, _I64, _P]),
     "recache_attend_prefill_history": (C.c_int, [_P, _P, _P, _P, _P, _P, _I32, _I32, _I32, _P, _P, _P, _I64, _P, _P,
                                                  _I64, _P, _P, _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
@@ -259,6 +261,28 @@ class ReCache:
                                              k_route.shape[0], _ptr(k_conv_out), _ptr(v_conv_out), _ptr(out), oc,
                                              _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_attend_prefill")
+        return out, k_conv_out, v_conv_out
+
+    def attend_prefill_gather(self, q, k_conv, v_conv, cu_q, q_pos0, max_q, k_cache, v_cache, route_idx, route_cu,
+                              k_conv_out=None, v_conv_out=None, out=None, out_dtype=None, workspace=None):
+        """recache_attend_prefill_gather: the route rows are read from the resource cache [G,pool,d]
+        through route_idx (index-only compaction).  Returns (o, k_conv_out, v_conv_out)."""
+        n_req = cu_q.numel() - 1
+        total_q = q.shape[0]
+        g, d = k_conv.shape[1], k_conv.shape[2]
+        od, oc = self._out_code(out_dtype)
+        if out is None:
+            out = torch.empty(q.shape, dtype=od, device=q.device)
+        if k_conv_out is None:
+            k_conv_out = torch.empty((g, total_q, d), dtype=k_conv.dtype, device=q.device)
+        if v_conv_out is None:
+            v_conv_out = torch.empty((g, total_q, d), dtype=k_conv.dtype, device=q.device)
+        ws = workspace if workspace is not None else self.workspace(self.prefill_workspace_bytes(n_req, total_q, max_q))
+        st = self.lib.recache_attend_prefill_gather(
+            self.h, _ptr(q), _ptr(k_conv), _ptr(v_conv), _ptr(cu_q), _ptr(q_pos0), n_req, total_q, int(max_q),
+            _ptr(k_cache), _ptr(v_cache), k_cache.shape[1], _ptr(route_idx), _ptr(route_cu), route_idx.numel(),
+            _ptr(k_conv_out), _ptr(v_conv_out), _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
+        self._check(st, "recache_attend_prefill_gather")
         return out, k_conv_out, v_conv_out
 
     def attend_prefill_history(self, q, k_conv, v_conv, cu_q, q_pos0, max_q, k_route, v_route, route_cu,

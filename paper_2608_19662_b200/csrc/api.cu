@@ -239,7 +239,9 @@ static recache_status prefill_impl(recache_ctx* ctx, const void* q, const void* 
                                    int32_t max_q, const void* k_route, const void* v_route, const int32_t* route_cu,
                                    int64_t route_rows, void* k_conv_out, void* v_conv_out, int64_t conv_rows,
                                    const int32_t* conv_slot, const int32_t* hist_len, void* out_o, int32_t out_dtype,
-                                   void* workspace, int64_t workspace_bytes, void* stream) {
+                                   void* workspace, int64_t workspace_bytes, void* stream,
+                                   const void* k_cache = nullptr, const void* v_cache = nullptr,
+                                   int64_t pool_tokens = 0, const int32_t* route_idx = nullptr) {
   if (!ctx) return RECACHE_EINVAL;
   RC_REQUIRE(n_requests >= 0 && total_q >= 0 && max_q >= 0 && route_rows >= 0 && conv_rows >= 0, RECACHE_EINVAL,
              "prefill: negative size");
@@ -247,7 +249,7 @@ static recache_status prefill_impl(recache_ctx* ctx, const void* q, const void* 
   if (n_requests == 0 || total_q == 0) return RECACHE_OK;
   RC_REQUIRE(q && k_conv && v_conv && cu_q && q_pos0 && route_cu && k_conv_out && v_conv_out && out_o,
              RECACHE_EINVAL, "prefill: null pointer");
-  RC_REQUIRE(route_rows == 0 || (k_route && v_route), RECACHE_EINVAL, "prefill: null route KV");
+  RC_REQUIRE(route_rows == 0 || (k_route && v_route) || route_idx, RECACHE_EINVAL, "prefill: null route KV");
   RC_REQUIRE(aligned16(q) && aligned16(k_conv) && aligned16(v_conv) && aligned16(k_route) && aligned16(v_route) &&
                  aligned16(k_conv_out) && aligned16(v_conv_out) && aligned16(out_o), RECACHE_EINVAL,
              "prefill: tensors must be 16-byte aligned");
@@ -262,6 +264,7 @@ static recache_status prefill_impl(recache_ctx* ctx, const void* q, const void* 
   RC_CUDA(rc_launch_rope_store(ctx, ra, st), "prefill: rope/store launch");
   PrefillArgs pa{q, out_o, out_dtype, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
                  route_rows, k_conv_out, v_conv_out, workspace, workspace_bytes, conv_rows, conv_slot, hist_len};
+  pa.k_cache = k_cache; pa.v_cache = v_cache; pa.pool_tokens = pool_tokens; pa.route_idx = route_idx;
   RC_CUDA(rc_launch_prefill_attn(ctx, pa, st), "prefill: attention launch");
   return RECACHE_OK;
 }
@@ -290,6 +293,25 @@ recache_status recache_attend_prefill_history(recache_ctx* ctx, const void* q, c
   return prefill_impl(ctx, q, k_conv, v_conv, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
                       route_rows, k_conv_cache, v_conv_cache, cache_rows, conv_slot, hist_len, out_o, out_dtype,
                       workspace, workspace_bytes, stream);
+}
+
+recache_status recache_attend_prefill_gather(recache_ctx* ctx, const void* q, const void* k_conv, const void* v_conv,
+                                             const int32_t* cu_q, const int32_t* q_pos0, int32_t n_requests,
+                                             int32_t total_q, int32_t max_q, const void* k_cache,
+                                             const void* v_cache, int64_t pool_tokens, const int32_t* route_idx,
+                                             const int32_t* route_cu, int64_t route_rows, void* k_conv_out,
+                                             void* v_conv_out, void* out_o, int32_t out_dtype, void* workspace,
+                                             int64_t workspace_bytes, void* stream) {
+  if (!ctx) return RECACHE_EINVAL;
+  RC_REQUIRE(rc_tc_supported(ctx), RECACHE_EUNSUPPORTED,
+             "prefill_gather: needs a bf16 context with head_dim 128 and 2, 4 or 8 query heads per KV head");
+  RC_REQUIRE(pool_tokens >= 0 && route_rows >= 0, RECACHE_EINVAL, "prefill_gather: negative size");
+  RC_REQUIRE(n_requests == 0 || total_q == 0 || (k_cache && v_cache && route_idx), RECACHE_EINVAL,
+             "prefill_gather: null cache / route_idx");
+  RC_REQUIRE(aligned16(k_cache) && aligned16(v_cache), RECACHE_EINVAL, "prefill_gather: caches must be 16-byte aligned");
+  return prefill_impl(ctx, q, k_conv, v_conv, cu_q, q_pos0, n_requests, total_q, max_q, nullptr, nullptr, route_cu,
+                      route_rows, k_conv_out, v_conv_out, (int64_t)total_q, nullptr, nullptr, out_o, out_dtype,
+                      workspace, workspace_bytes, stream, k_cache, v_cache, pool_tokens, route_idx);
 }
 
 recache_status recache_attend_decode(recache_ctx* ctx, const void* q, const int32_t* q_pos, int32_t batch,

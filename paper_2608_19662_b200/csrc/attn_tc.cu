@@ -11,7 +11,7 @@
 //   warp  8      TMA producer         warp  9    tcgen05.mma issuer (+ TMEM alloc)
 //   warp  10     scheduler: draws work items from a global counter and publishes
 //                them through a two-slot ring in shared memory
-//   warp  11     idle (completes the third warpgroup)
+//   warp  11     idle (completes the third warpgroup); V-tile producer in gather mode
 //   warps 12-15  epilogue: O of a finished tile goes from tensor memory to HBM
 //                while the softmax warps already rotate the next item's Q
 // setmaxnreg moves registers from warps 8-15 to the two softmax warpgroups,
@@ -71,6 +71,8 @@ constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long i
 struct TcParams {
   const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter, header[2] = order[] is valid
   const int32_t* order;                 // work indices, heaviest first (launches of at most SORT_MAX work items)
+  // gather mode: route row n of group g is row route_idx[n] of gather_k / gather_v ([G][pool_tokens][128] bf16)
+  const uint8_t* gather_k; const uint8_t* gather_v; const int32_t* route_idx; int64_t pool_tokens;
   const int32_t* cu; const int32_t* pos0; const int32_t* slot; const int32_t* route_cu; const int32_t* hist;
   int n_seq, G, Hq, s;
   int prefix_len;   // > 0: every sequence sees rows g*prefix_len .. of the "route" tensors (shared prefix)
@@ -125,6 +127,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(src_bytes) : "memory");
+}
+// one arrival on the barrier once all earlier cp.async of this thread have landed (the barrier's
+// expected count already includes it)
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 // plain bulk copy global -> shared (16-byte aligned, size a multiple of 16)
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -376,7 +387,7 @@ __global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int t
 // items through a two-slot ring in shared memory.
 // The next item's Q load, Q rotation and first K/V tiles overlap the current
 // item's last tiles and its epilogue.  Barrier phases run on across items.
-template <typename TO, bool ROT_SMEM>
+template <typename TO, bool ROT_SMEM, bool GATHER>
 __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                               const __grid_constant__ CUtensorMap tm_ks,
                                                               const __grid_constant__ CUtensorMap tm_vs,
@@ -402,13 +413,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QREADY + 0), 128); mbar_init(bar(B_QREADY + 1), 128);
     mbar_init(bar(B_QEMPTY), 1);
-    for (int i = 0; i < NSTAGE; ++i) {
-      mbar_init(bar(B_KFULL + i), 1); mbar_init(bar(B_KEMPTY + i), 1);
-      mbar_init(bar(B_VFULL + i), 1); mbar_init(bar(B_VEMPTY + i), 1);
+    for (int i = 0; i < NSTAGE; ++i) {   // gather mode: a whole warp fills a K (or V) stage and every lane arrives
+      mbar_init(bar(B_KFULL + i), GATHER ? 32 : 1); mbar_init(bar(B_KEMPTY + i), 1);
+      mbar_init(bar(B_VFULL + i), GATHER ? 32 : 1); mbar_init(bar(B_VEMPTY + i), 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1); mbar_init(bar(B_PREADY + x), 128); mbar_init(bar(B_ODONE + x), 1);
-      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 386);   // producer + MMA + 256 softmax + 128 epilogue threads
+      // producer (two of them in gather mode) + MMA + 256 softmax + 128 epilogue threads
+      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), GATHER ? 387 : 386);
       mbar_init(bar(B_LREADY + x), 128); mbar_init(bar(B_ODRAIN + x), 128); mbar_init(bar(B_PHALF + x), 128);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -533,6 +545,87 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       }
     }
     __syncwarp();
+  } else if (GATHER && (warp == 8 || warp == 11)) {
+    // ===================== producers, gather mode =====================
+    // Route tiles are not packed anywhere: row n of the route is row route_idx[n] of the resource
+    // cache.  Warp 8 fills the K stages (and loads Q), warp 11 the V stages: 16-byte asynchronous
+    // copies straight into the swizzled tile layout, 64 per lane and tile; every lane's arrival on
+    // the stage's barrier fires when its copies have landed, and the MMA warp puts a proxy fence
+    // between that and the tensor core's reads.  The conversation's own tiles still come by TMA.
+    const bool is_k = warp == 8;
+    const uint8_t* src_base = is_k ? p.gather_k : p.gather_v;
+    const uint32_t stage0 = sm + (is_k ? SM_K : SM_V);
+    const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
+    const CUtensorMap* tm_self = is_k ? &tm_ks : &tm_vs;
+    Item it;
+    uint32_t kv_n = 0;
+    for (uint32_t item_n = 0;; ++item_n) {
+      fetch_item(item_n, it, false);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_IEMPTY + (item_n & 1u)));
+      if (it.n_tiles < 0) break;
+      if (is_k && lane == 0) {
+        // Q tiles: free once the previous item's last S = Q K^T has completed
+        mbar_wait(bar(B_QEMPTY), (item_n & 1u) ^ 1u, abort_flag, p.status);
+        uint32_t rot_bytes = 0;
+        const int pos_start = it.pos0 + it.tok0;
+        if (ROT_SMEM) {
+          const int rows = min(2 * TQ, p.max_pos - pos_start);
+          if (pos_start >= 0 && rows > 0) rot_bytes = (uint32_t)rows * 256u;
+        }
+        mbar_expect_tx(bar(B_QFULL), 2 * TILE_BYTES + 2 * rot_bytes);
+        for (int x = 0; x < 2; ++x)
+          for (int kc = 0; kc < 2; ++kc)
+            tma_load_3d(sm + SM_Q + x * TILE_BYTES + kc * BOX_BYTES, &tm_q, bar(B_QFULL), kc * 64, it.g * s,
+                        it.seq0 + it.tok0 + x * TQ);
+        if (rot_bytes) {
+          bulk_load(sm + SM_ROT, p.cos_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
+          bulk_load(sm + SM_ROT + ROT_BYTES, p.sin_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
+        }
+      }
+      __syncwarp();
+      for (int i = 0; i < it.n_tiles; ++i, ++kv_n) {
+        const int st = kv_n % NSTAGE;
+        const uint32_t ph = (kv_n / NSTAGE) & 1u;
+        mbar_wait(bar(b_empty + st), ph ^ 1u, abort_flag, p.status);
+        if (i < it.nA) {
+          const int r0 = it.rA0 + i * TILE_N, cnt = min(TILE_N, it.lenA - i * TILE_N);
+          const uint8_t* grp = src_base + (int64_t)it.g * p.pool_tokens * 256;
+          const uint32_t dst0 = stage0 + st * TILE_BYTES;
+          // the tile's 128 indices: four coalesced loads per lane, handed round by shuffles
+          int idx4[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int r = lane + 32 * j;
+            int idx = r < cnt ? p.route_idx[r0 + r] : -1;
+            if (r < cnt && (idx < 0 || idx >= p.pool_tokens)) { rc_set_status(p.status, RECACHE_DEV_BAD_SLOT); idx = -1; }
+            idx4[j] = idx;
+          }
+          const int hi = lane >> 4, c = lane & 15;
+          const uint32_t dst_c = dst0 + (c >> 3) * BOX_BYTES;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+#pragma unroll 4
+            for (int kk = 0; kk < 16; ++kk) {
+              const int r = 32 * j + 2 * kk + hi;               // piece (row r, 16-byte chunk c)
+              const int idx = __shfl_sync(0xffffffffu, idx4[j], 2 * kk + hi);
+              cp_async16(dst_c + r * 128 + (((c & 7) ^ (r & 7)) << 4), grp + (int64_t)max(idx, 0) * 256 + c * 16,
+                         idx >= 0 ? 16u : 0u);
+            }
+          }
+          cp_async_arrive(bar(b_full + st));
+        } else {
+          const int row = (int)((int64_t)it.g * p.self_rows + it.base) + (i - it.nA) * TILE_N;
+          if (lane == 0) {
+            mbar_expect_tx(bar(b_full + st), TILE_BYTES);
+            for (int kc = 0; kc < 2; ++kc)
+              tma_load_2d(stage0 + st * TILE_BYTES + kc * BOX_BYTES, tm_self, bar(b_full + st), kc * 64, row);
+          } else {
+            mbar_arrive(bar(b_full + st));
+          }
+        }
+      }
+    }
   } else if (warp == 8) {
     // ===================== TMA producer =====================
     if (lane == 0) {
@@ -613,6 +706,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       // each query tile starts as soon as its own half of Q has been rotated
       mbar_wait(bar(B_QREADY + 0), item_n & 1u, abort_flag, p.status);
       mbar_wait(bar(B_KFULL + kv_n % NSTAGE), (kv_n / NSTAGE) & 1u, abort_flag, p.status);
+      if (GATHER) fence_async_smem();   // the tile may have been written by cp.async (generic proxy)
       tc_fence_after();
       const int st0 = kv_n % NSTAGE;
       if (issuer) { issue_qk(0, st0); tc_commit(bar(B_SFULL + 0)); }
@@ -634,6 +728,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const int vis_rows = i < nA ? seg_rows : kv_end - (i - nA) * TILE_N;
         const int ksteps = (min(vis_rows, TILE_N) + 15) >> 4;
         mbar_wait(bar(B_VFULL + st), ph, abort_flag, p.status);
+        if (GATHER) fence_async_smem();
         if (seg_rows < ksteps * 16) {
           // rows past the segment hold whatever follows it in memory: zero them, 0 * NaN would poison O
           uint8_t* vb = sm_gen + SM_V + st * TILE_BYTES;
@@ -658,6 +753,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         if (issuer) { issue_pv(0, st, 4, ksteps, false); if (!more) tc_commit(bar(B_ODONE + 0)); }
         if (more) {
           mbar_wait(bar(B_KFULL + st1), ph1, abort_flag, p.status);
+          if (GATHER) fence_async_smem();
           tc_fence_after();
           if (issuer) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
         }
@@ -940,7 +1036,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   if (!map_q(&tq, a.q, (uint64_t)a.total, Hq, s) || !map_rows(&tks, a.k_self, self_total) ||
       !map_rows(&tvs, a.v_self, self_total))
     return cudaErrorInvalidValue;
-  const bool has_route = (a.route_cu != nullptr || a.prefix_len > 0) && a.route_rows > 0;
+  const bool has_route = (a.route_cu != nullptr || a.prefix_len > 0) && a.route_rows > 0 && a.route_idx == nullptr;
   if (!map_rows(&tkr, has_route ? a.k_route : a.k_self, has_route ? (uint64_t)a.route_rows : self_total) ||
       !map_rows(&tvr, has_route ? a.v_route : a.v_self, has_route ? (uint64_t)a.route_rows : self_total))
     return cudaErrorInvalidValue;
@@ -954,6 +1050,9 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)ctx->desc.head_dim));
   p.status = ctx->status;
   p.order = order;
+  const bool gather = a.route_idx != nullptr;
+  p.gather_k = (const uint8_t*)a.k_cache; p.gather_v = (const uint8_t*)a.v_cache; p.route_idx = a.route_idx;
+  p.pool_tokens = a.pool_tokens;
   {
     RcLaunchScope scope(ctx, RC_K_TILE_PLAN, st);
     tile_plan_kernel<<<1, 1024, 0, st>>>(p, tc_tok_per_cta(ctx), n_levels, items, level_off, order, (int)max_items);
@@ -966,8 +1065,13 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
     kernel<<<grid, NTHREADS, SM_ALLOC, st>>>(tq, tks, tvs, tkr, tvr, p);
   };
   const bool f32 = a.out_dtype == RECACHE_F32, rot = s >= 4;   // 2 * 128 / s <= 64 positions fit the staging area
-  if (f32) { if (rot) launch(attn_tc_kernel<float, true>); else launch(attn_tc_kernel<float, false>); }
-  else { if (rot) launch(attn_tc_kernel<__nv_bfloat16, true>); else launch(attn_tc_kernel<__nv_bfloat16, false>); }
+  if (gather) {
+    if (f32) { if (rot) launch(attn_tc_kernel<float, true, true>); else launch(attn_tc_kernel<float, false, true>); }
+    else { if (rot) launch(attn_tc_kernel<__nv_bfloat16, true, true>); else launch(attn_tc_kernel<__nv_bfloat16, false, true>); }
+  } else {
+    if (f32) { if (rot) launch(attn_tc_kernel<float, true, false>); else launch(attn_tc_kernel<float, false, false>); }
+    else { if (rot) launch(attn_tc_kernel<__nv_bfloat16, true, false>); else launch(attn_tc_kernel<__nv_bfloat16, false, false>); }
+  }
   return cudaGetLastError();
 }
 

@@ -155,6 +155,8 @@ struct PrefillArgs {
   int64_t conv_rows;                        // rows per group of k_conv / v_conv
   const int32_t* conv_slot = nullptr;       // first row of each request's region (null: cu_q[b])
   const int32_t* hist = nullptr;            // earlier-turn rows at the start of that region (null: 0)
+  // gather mode: see TcAttnArgs
+  const void* k_cache = nullptr; const void* v_cache = nullptr; int64_t pool_tokens = 0; const int32_t* route_idx = nullptr;
 };
 int64_t rc_encode_workspace_bytes(const recache_ctx* ctx, int n_res, int total, int max_len);
 int64_t rc_prefill_workspace_bytes(const recache_ctx* ctx, int n_req, int total_q, int max_q);
@@ -174,6 +176,9 @@ struct TcAttnArgs {
   void* workspace;
   int prefix_len;   // > 0 (route_cu null): all sequences see rows g*prefix_len .. of k_route/v_route ([G*prefix_len][128])
   const int32_t* hist = nullptr;   // rows preceding each sequence's own tokens in the self part (earlier turns), all visible
+  // gather mode (route_idx != null): route rows are rows route_idx[.] of group g in k_cache / v_cache
+  // ([G][pool_tokens][128]); k_route / v_route are unused
+  const void* k_cache = nullptr; const void* v_cache = nullptr; int64_t pool_tokens = 0; const int32_t* route_idx = nullptr;
 };
 bool rc_tc_supported(const recache_ctx* ctx);
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);

@@ -31,6 +31,7 @@ cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a,
   if (rc_tc_supported(ctx)) {
     TcAttnArgs t{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.max_q, a.pos0, a.conv_slot, a.k_conv, a.v_conv,
                  a.conv_rows, a.k_route, a.v_route, a.route_cu, a.route_rows, a.workspace, 0, a.hist};
+    t.k_cache = a.k_cache; t.v_cache = a.v_cache; t.pool_tokens = a.pool_tokens; t.route_idx = a.route_idx;
     return rc_launch_attn_tc(ctx, t, st);
   }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, a.conv_slot, a.k_conv, a.v_conv,
