@@ -601,16 +601,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             if (r < cnt && (idx < 0 || idx >= p.pool_tokens)) { rc_set_status(p.status, RECACHE_DEV_BAD_SLOT); idx = -1; }
             idx4[j] = idx;
           }
+          // piece (row r = 32 j + 2 kk + hi, 16-byte chunk c): the swizzle term only depends on kk & 3
           const int hi = lane >> 4, c = lane & 15;
-          const uint32_t dst_c = dst0 + (c >> 3) * BOX_BYTES;
+          const uint32_t dst_l = dst0 + (c >> 3) * BOX_BYTES + hi * 128;
+          uint32_t sw[4];
+#pragma unroll
+          for (int m = 0; m < 4; ++m) sw[m] = (uint32_t)(((c & 7) ^ ((2 * m + hi) & 7)) << 4);
+          const uint8_t* src_l = grp + c * 16;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-#pragma unroll 4
+#pragma unroll
             for (int kk = 0; kk < 16; ++kk) {
-              const int r = 32 * j + 2 * kk + hi;               // piece (row r, 16-byte chunk c)
               const int idx = __shfl_sync(0xffffffffu, idx4[j], 2 * kk + hi);
-              cp_async16(dst_c + r * 128 + (((c & 7) ^ (r & 7)) << 4), grp + (int64_t)max(idx, 0) * 256 + c * 16,
-                         idx >= 0 ? 16u : 0u);
+              cp_async16(dst_l + (32 * j + 2 * kk) * 128 + sw[kk & 3], src_l + (int64_t)max(idx, 0) * 256, idx >= 0 ? 16u : 0u);
             }
           }
           cp_async_arrive(bar(b_full + st));
