@@ -689,12 +689,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         mma_ss(dst, qa + off, ka + off, IDESC_QK, j > 0);
       }
     };
+    // K steps k0 .. ksteps-1 of O += P V (16 keys each); a full half (4 steps) is the common case
     auto issue_pv = [&](int x, int st, int k0, int ksteps, bool first) {
       const uint64_t va = d_v + st * (TILE_BYTES >> 4);
       const uint32_t dst = tmem + COL_O + 128 * x, src = tmem + COL_S + 128 * x;
-#pragma unroll 4
-      for (int j = k0; j < ksteps; ++j)
-        mma_ts(dst, src + 8 * j, va + j * (2048 >> 4), IDESC_PV, (!first || j > 0) ? 1u : 0u);
+      if (ksteps - k0 == 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          mma_ts(dst, src + 8 * (k0 + j), va + (k0 + j) * (2048 >> 4), IDESC_PV, (!first || j > 0) ? 1u : 0u);
+      } else {
+#pragma unroll 1
+        for (int j = k0; j < ksteps; ++j)
+          mma_ts(dst, src + 8 * j, va + j * (2048 >> 4), IDESC_PV, (!first || j > k0) ? 1u : 0u);
+      }
     };
     Item it;
     uint32_t kv_n = 0, cnt[2] = {0, 0};   // K/V tiles, tiles per query tile so far
