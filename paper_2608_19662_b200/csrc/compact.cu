@@ -83,8 +83,10 @@ __global__ void __launch_bounds__(1024) compact_plan_kernel(
     const int32_t* __restrict__ free_pages, int64_t n_free_pages, int64_t n_pool_pages,
     int32_t* status) {
   __shared__ int ws[1024 / 32 + 1];
+  __shared__ int wlen_sh[32];
   __shared__ int carry_rows, carry_pages;
   const int n_routes = n_requests * G;
+  const bool warp_per_route = n_routes <= 32;
   if (threadIdx.x == 0) { carry_rows = 0; carry_pages = 0; }
   __syncthreads();
   for (int r0 = 0; r0 < n_routes; r0 += blockDim.x) {
@@ -95,12 +97,41 @@ __global__ void __launch_bounds__(1024) compact_plan_kernel(
       const int a = res_off[b], e = res_off[b + 1];
       if (a < 0 || e < a || e > total_listed) {
         rc_set_status(status, RECACHE_DEV_BAD_SEQLENS);
-      } else {
+      } else if (!warp_per_route) {
         for (int r = a; r < e; ++r) {
           res_route_off[(int64_t)g * total_listed + r] = len;
           if (vis[(int64_t)g * total_listed + r]) len += kept[r];
         }
       }
+    }
+    if (warp_per_route) {
+      // few routes, many resources each (a prefill): warp w walks route w's list 32 resources at a
+      // time (independent loads, one warp scan per chunk), then hands the length to thread w
+      const int lane = threadIdx.x & 31, wr = r0 + (threadIdx.x >> 5);
+      int wlen = 0;
+      if (wr < n_routes) {
+        const int b = wr / G, g = wr % G;
+        const int a = res_off[b], e = res_off[b + 1];
+        if (a >= 0 && e >= a && e <= total_listed) {
+          for (int c0 = a; c0 < e; c0 += 32) {
+            const int r = c0 + lane;
+            int v = 0;
+            if (r < e && vis[(int64_t)g * total_listed + r]) v = kept[r];
+            int incl = v;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+              const int u = __shfl_up_sync(0xffffffffu, incl, off);
+              if (lane >= off) incl += u;
+            }
+            if (r < e) res_route_off[(int64_t)g * total_listed + r] = wlen + incl - v;
+            wlen += __shfl_sync(0xffffffffu, incl, 31);
+          }
+        }
+      }
+      if (lane == 0) wlen_sh[threadIdx.x >> 5] = wlen;
+      __syncthreads();
+      if (route < n_routes && threadIdx.x < 32) len = wlen_sh[threadIdx.x];
+      __syncthreads();
     }
     const int pages = (mode == RECACHE_PAGED) ? (len + page_tokens - 1) / page_tokens : 0;
     int tot_rows, tot_pages;
