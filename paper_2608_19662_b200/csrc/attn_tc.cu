@@ -466,13 +466,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     for (uint32_t item_n = 0; it.n_tiles > 0; ++item_n) {
       fetch_item(item_n + 1, nx, true);
       // The stores below and the rotation of the next item's Q go through the same load/store
-      // path, and only the rotation is urgent: let it finish first.  (O is not needed back before
-      // the next item's first P V, a whole softmax later.)
-      if (nx.n_tiles > 0) {
-        mbar_wait(bar(B_QREADY + 0), (item_n + 1u) & 1u, abort_flag, p.status);
-        mbar_wait(bar(B_QREADY + 1), (item_n + 1u) & 1u, abort_flag, p.status);
-      }
+      // path, and the rotation is the urgent one: a tile's O is written back once the same tile's
+      // next Q has been rotated.  (O is not needed back before the next item's first P V, a whole
+      // softmax later; tile B's rotation finishes after tile A's, so tile A is not held up by it.)
       for (int x = 0; x < 2; ++x) {
+        if (nx.n_tiles > 0) mbar_wait(bar(B_QREADY + x), (item_n + 1u) & 1u, abort_flag, p.status);
         if (x == 1 && !it.b_valid) continue;
         mbar_wait(bar(B_LREADY + x), done[x] & 1u, abort_flag, p.status);
         mbar_wait(bar(B_ODONE + x), done[x] & 1u, abort_flag, p.status);
