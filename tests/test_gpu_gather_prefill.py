@@ -25,16 +25,17 @@ def _index_only(rc, pool, req, kc, vc):
     return r_cu, r_idx
 
 
-def test_gather_prefill_equals_packed_prefill_and_oracle():
+@pytest.mark.parametrize("sh", [wl.QWEN3_4B, wl.Shape(16, 8, 128, 1e6, "bf16"), wl.Shape(16, 2, 128, 1e4, "bf16")],
+                         ids=["4_per_group", "2_per_group", "8_per_group"])
+def test_gather_prefill_equals_packed_prefill_and_oracle(sh):
     """Several requests with ragged routes (tail tiles, an empty route) and ragged lengths."""
-    sh = wl.QWEN3_4B
     g = sh.n_kv_heads
     rng = np.random.default_rng(31)
     lens = [300, 77, 130, 512, 45, 260]
     pool = wl.pack_resources(sh, 31, lens, wl.keep_mask_spans(rng, lens))
     res_lists = [[0, 3, 5], [1, 2], [4, 0, 2, 3]]
     vis = [wl.routes_random(rng, g, len(l), 0.5) for l in res_lists]
-    vis[1][2, :] = 0                                     # an empty route: plain causal attention for that group
+    vis[1][g - 1, :] = 0                                 # an empty route: plain causal attention for that group
     req = wl.make_requests(sh, 32, pool, res_lists, vis, [150, 64, 333])
     rc = make_ctx(sh, max_pos=4096)
     _, kc, vc = gpu_encode(rc, pool)
