@@ -11,7 +11,7 @@
 //   warp  8      TMA producer         warp  9    tcgen05.mma issuer (+ TMEM alloc)
 //   warp  10     scheduler: draws work items from a global counter and publishes
 //                them through a two-slot ring in shared memory
-//   warp  11     idle (completes the third warpgroup); V-tile producer in gather mode
+//   warp  11     idle (completes the third warpgroup)
 //   warps 12-15  epilogue: O of a finished tile goes from tensor memory to HBM
 //                while the softmax warps already rotate the next item's Q
 // setmaxnreg moves registers from warps 8-15 to the two softmax warpgroups,
@@ -413,14 +413,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     mbar_init(bar(B_QFULL), 1);
     mbar_init(bar(B_QREADY + 0), 128); mbar_init(bar(B_QREADY + 1), 128);
     mbar_init(bar(B_QEMPTY), 1);
-    for (int i = 0; i < NSTAGE; ++i) {   // gather mode: a whole warp fills a K (or V) stage and every lane arrives
-      mbar_init(bar(B_KFULL + i), GATHER ? 32 : 1); mbar_init(bar(B_KEMPTY + i), 1);
-      mbar_init(bar(B_VFULL + i), GATHER ? 32 : 1); mbar_init(bar(B_VEMPTY + i), 1);
+    for (int i = 0; i < NSTAGE; ++i) {   // gather mode: the 128 epilogue lanes and the TMA producer arrive on every stage
+      mbar_init(bar(B_KFULL + i), GATHER ? 129 : 1); mbar_init(bar(B_KEMPTY + i), 1);
+      mbar_init(bar(B_VFULL + i), GATHER ? 129 : 1); mbar_init(bar(B_VEMPTY + i), 1);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(bar(B_SFULL + x), 1); mbar_init(bar(B_PREADY + x), 128); mbar_init(bar(B_ODONE + x), 1);
-      // producer (two of them in gather mode) + MMA + 256 softmax + 128 epilogue threads
-      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), GATHER ? 387 : 386);
+      // producer + MMA + 256 softmax + 128 epilogue threads
+      mbar_init(bar(B_IFULL + x), 1); mbar_init(bar(B_IEMPTY + x), 386);
       mbar_init(bar(B_LREADY + x), 128); mbar_init(bar(B_ODRAIN + x), 128); mbar_init(bar(B_PHALF + x), 128);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -463,7 +463,51 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     Item it, nx;
     uint32_t done[2] = {0, 0};
     fetch_item(0, it, true);
+    uint32_t kv_n = 0;
     for (uint32_t item_n = 0; it.n_tiles > 0; ++item_n) {
+      if (GATHER) {
+        // Gather mode: these 128 lanes also fill the route tiles of the item.  Row n of the route is
+        // row route_idx[n] of the resource cache: warp w takes rows 32 w .. 32 w + 31 of a tile, one
+        // index per lane handed round by shuffles, 16 16-byte asynchronous copies per lane straight
+        // to the swizzled positions of a TMA tile (zero-fill past the route's end).  A lane's arrival
+        // fires when its copies have landed; the MMA warp puts a proxy fence before the reads.
+        const int w = warp & 3, hi = lane >> 4, c = lane & 15;
+        uint32_t sw[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) sw[m] = (uint32_t)(((c & 7) ^ ((2 * m + hi) & 7)) << 4);
+        for (int i = 0; i < it.n_tiles; ++i) {
+          const uint32_t n = kv_n + (uint32_t)i;
+          const int st = n % NSTAGE;
+          const uint32_t ph = (n / NSTAGE) & 1u;
+          const bool route = i < it.nA;
+          int idx = -1;
+          if (route) {
+            const int r = 32 * w + lane, cnt = min(TILE_N, it.lenA - i * TILE_N);
+            if (r < cnt) {
+              idx = p.route_idx[it.rA0 + i * TILE_N + r];
+              if (idx < 0 || idx >= p.pool_tokens) { rc_set_status(p.status, RECACHE_DEV_BAD_SLOT); idx = -1; }
+            }
+          }
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv) {
+            const int b_full = kv ? B_VFULL : B_KFULL, b_empty = kv ? B_VEMPTY : B_KEMPTY;
+            mbar_wait(bar(b_empty + st), ph ^ 1u, abort_flag, p.status);
+            if (route) {
+              const uint8_t* src_l = (kv ? p.gather_v : p.gather_k) + (int64_t)it.g * p.pool_tokens * 256 + c * 16;
+              const uint32_t dst_l = sm + (kv ? SM_V : SM_K) + st * TILE_BYTES + (c >> 3) * BOX_BYTES + (32 * w + hi) * 128;
+#pragma unroll
+              for (int kk = 0; kk < 16; ++kk) {
+                const int ix = __shfl_sync(0xffffffffu, idx, 2 * kk + hi);
+                cp_async16(dst_l + 2 * kk * 128 + sw[kk & 3], src_l + (int64_t)max(ix, 0) * 256, ix >= 0 ? 16u : 0u);
+              }
+              cp_async_arrive(bar(b_full + st));
+            } else {
+              mbar_arrive(bar(b_full + st));
+            }
+          }
+        }
+        kv_n += (uint32_t)it.n_tiles;
+      }
       fetch_item(item_n + 1, nx, true);
       // The stores below and the rotation of the next item's Q go through the same load/store
       // path, and the rotation is the urgent one: a tile's O is written back once the same tile's
@@ -543,90 +587,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       }
     }
     __syncwarp();
-  } else if (GATHER && (warp == 8 || warp == 11)) {
-    // ===================== producers, gather mode =====================
-    // Route tiles are not packed anywhere: row n of the route is row route_idx[n] of the resource
-    // cache.  Warp 8 fills the K stages (and loads Q), warp 11 the V stages: 16-byte asynchronous
-    // copies straight into the swizzled tile layout, 64 per lane and tile; every lane's arrival on
-    // the stage's barrier fires when its copies have landed, and the MMA warp puts a proxy fence
-    // between that and the tensor core's reads.  The conversation's own tiles still come by TMA.
-    const bool is_k = warp == 8;
-    const uint8_t* src_base = is_k ? p.gather_k : p.gather_v;
-    const uint32_t stage0 = sm + (is_k ? SM_K : SM_V);
-    const int b_full = is_k ? B_KFULL : B_VFULL, b_empty = is_k ? B_KEMPTY : B_VEMPTY;
-    const CUtensorMap* tm_self = is_k ? &tm_ks : &tm_vs;
-    Item it;
-    uint32_t kv_n = 0;
-    for (uint32_t item_n = 0;; ++item_n) {
-      fetch_item(item_n, it, false);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_IEMPTY + (item_n & 1u)));
-      if (it.n_tiles < 0) break;
-      if (is_k && lane == 0) {
-        // Q tiles: free once the previous item's last S = Q K^T has completed
-        mbar_wait(bar(B_QEMPTY), (item_n & 1u) ^ 1u, abort_flag, p.status);
-        uint32_t rot_bytes = 0;
-        const int pos_start = it.pos0 + it.tok0;
-        if (ROT_SMEM) {
-          const int rows = min(2 * TQ, p.max_pos - pos_start);
-          if (pos_start >= 0 && rows > 0) rot_bytes = (uint32_t)rows * 256u;
-        }
-        mbar_expect_tx(bar(B_QFULL), 2 * TILE_BYTES + 2 * rot_bytes);
-        for (int x = 0; x < 2; ++x)
-          for (int kc = 0; kc < 2; ++kc)
-            tma_load_3d(sm + SM_Q + x * TILE_BYTES + kc * BOX_BYTES, &tm_q, bar(B_QFULL), kc * 64, it.g * s,
-                        it.seq0 + it.tok0 + x * TQ);
-        if (rot_bytes) {
-          bulk_load(sm + SM_ROT, p.cos_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
-          bulk_load(sm + SM_ROT + ROT_BYTES, p.sin_tab + (int64_t)pos_start * 64, rot_bytes, bar(B_QFULL));
-        }
-      }
-      __syncwarp();
-      for (int i = 0; i < it.n_tiles; ++i, ++kv_n) {
-        const int st = kv_n % NSTAGE;
-        const uint32_t ph = (kv_n / NSTAGE) & 1u;
-        mbar_wait(bar(b_empty + st), ph ^ 1u, abort_flag, p.status);
-        if (i < it.nA) {
-          const int r0 = it.rA0 + i * TILE_N, cnt = min(TILE_N, it.lenA - i * TILE_N);
-          const uint8_t* grp = src_base + (int64_t)it.g * p.pool_tokens * 256;
-          const uint32_t dst0 = stage0 + st * TILE_BYTES;
-          // the tile's 128 indices: four coalesced loads per lane, handed round by shuffles
-          int idx4[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int r = lane + 32 * j;
-            int idx = r < cnt ? p.route_idx[r0 + r] : -1;
-            if (r < cnt && (idx < 0 || idx >= p.pool_tokens)) { rc_set_status(p.status, RECACHE_DEV_BAD_SLOT); idx = -1; }
-            idx4[j] = idx;
-          }
-          // piece (row r = 32 j + 2 kk + hi, 16-byte chunk c): the swizzle term only depends on kk & 3
-          const int hi = lane >> 4, c = lane & 15;
-          const uint32_t dst_l = dst0 + (c >> 3) * BOX_BYTES + hi * 128;
-          uint32_t sw[4];
-#pragma unroll
-          for (int m = 0; m < 4; ++m) sw[m] = (uint32_t)(((c & 7) ^ ((2 * m + hi) & 7)) << 4);
-          const uint8_t* src_l = grp + c * 16;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-#pragma unroll
-            for (int kk = 0; kk < 16; ++kk) {
-              const int idx = __shfl_sync(0xffffffffu, idx4[j], 2 * kk + hi);
-              cp_async16(dst_l + (32 * j + 2 * kk) * 128 + sw[kk & 3], src_l + (int64_t)max(idx, 0) * 256, idx >= 0 ? 16u : 0u);
-            }
-          }
-          cp_async_arrive(bar(b_full + st));
-        } else {
-          const int row = (int)((int64_t)it.g * p.self_rows + it.base) + (i - it.nA) * TILE_N;
-          if (lane == 0) {
-            mbar_expect_tx(bar(b_full + st), TILE_BYTES);
-            for (int kc = 0; kc < 2; ++kc)
-              tma_load_2d(stage0 + st * TILE_BYTES + kc * BOX_BYTES, tm_self, bar(b_full + st), kc * 64, row);
-          } else {
-            mbar_arrive(bar(b_full + st));
-          }
-        }
-      }
-    }
   } else if (warp == 8) {
     // ===================== TMA producer =====================
     if (lane == 0) {
@@ -658,14 +618,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           const bool route = i < it.nA;
           const int row = route ? it.rA0 + i * TILE_N
                                 : (int)((int64_t)it.g * p.self_rows + it.base) + (i - it.nA) * TILE_N;
+          // (gather mode: a route tile is filled by the epilogue warps; every stage barrier expects
+          // their 128 arrivals plus one from here, whoever brings the data)
           mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, abort_flag, p.status);
-          mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
-          for (int kc = 0; kc < 2; ++kc)
-            tma_load_2d(sm + SM_K + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_kr : &tm_ks, bar(B_KFULL + st), kc * 64, row);
+          if (GATHER && route) {
+            mbar_arrive(bar(B_KFULL + st));
+          } else {
+            mbar_expect_tx(bar(B_KFULL + st), TILE_BYTES);
+            for (int kc = 0; kc < 2; ++kc)
+              tma_load_2d(sm + SM_K + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_kr : &tm_ks, bar(B_KFULL + st), kc * 64, row);
+          }
           mbar_wait(bar(B_VEMPTY + st), ph ^ 1u, abort_flag, p.status);
-          mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
-          for (int kc = 0; kc < 2; ++kc)
-            tma_load_2d(sm + SM_V + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_vr : &tm_vs, bar(B_VFULL + st), kc * 64, row);
+          if (GATHER && route) {
+            mbar_arrive(bar(B_VFULL + st));
+          } else {
+            mbar_expect_tx(bar(B_VFULL + st), TILE_BYTES);
+            for (int kc = 0; kc < 2; ++kc)
+              tma_load_2d(sm + SM_V + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_vr : &tm_vs, bar(B_VFULL + st), kc * 64, row);
+          }
         }
       }
     }
