@@ -204,6 +204,61 @@ class Runner:
         self.h_o_dec.copy_(self.o_dec, non_blocking=True)
 
 
+def other_workload_config3(device: int, peak_tf: float, iters: int = 20):
+    """One layer of the composition-reuse shape (64 pool resources U[150,1200] encoded once, 16 requests of
+    4-12 of them with 256-1024 query tokens): attention throughput of the encode and the prefill launch from
+    the library's event timer.  A side measurement: not part of `value`."""
+    from paper_2608_19662_b200 import PACKED, ReCache
+    pool = wl.config3_pool(layer=7)
+    req = wl.config3_requests(pool, layer=7)
+    sh = pool.shape
+    dev = torch.device("cuda", device)
+    g, d = sh.n_kv_heads, sh.head_dim
+    max_pos = int(max(req.q_pos0.max() + req.max_q, pool.max_len)) + 1
+    rc = ReCache(sh.n_q_heads, g, d, sh.rope_theta, sh.dtype, max_pos=max_pos, page_tokens=wl.PAGE_TOKENS, device=device)
+    t = lambda a: (torch.from_numpy(np.ascontiguousarray(a)) if isinstance(a, np.ndarray) else a).to(dev)
+    q, k, v, cu, slot, keep = t(pool.q), t(pool.k), t(pool.v), t(pool.cu_seqlens), t(pool.dst_slot), t(pool.keep)
+    res_off, res_slot, res_len, vis = t(req.res_off), t(req.res_slot), t(req.res_len), t(req.vis)
+    cq, ck, cv, cu_q, q_pos0 = t(req.q), t(req.k_conv), t(req.v_conv), t(req.cu_q), t(req.q_pos0)
+    kc = torch.empty((g, pool.pool_tokens, d), dtype=sh.torch_dtype, device=dev)
+    vc = torch.empty_like(kc)
+    o_enc = torch.empty((pool.total_tokens, sh.n_q_heads, d), dtype=sh.torch_dtype, device=dev)
+    n_routes = req.n_requests * g
+    cap = int(req.res_len.sum()) * g + 64
+    route_cu = torch.empty(n_routes + 1, dtype=torch.int32, device=dev)
+    route_idx = torch.empty(cap, dtype=torch.int32, device=dev)
+    k_route, v_route = torch.empty((cap, d), dtype=sh.torch_dtype, device=dev), torch.empty((cap, d), dtype=sh.torch_dtype, device=dev)
+    o_pre = torch.empty((req.total_q, sh.n_q_heads, d), dtype=sh.torch_dtype, device=dev)
+
+    def layer():
+        rc.encode_resources(q, k, v, cu, pool.max_len, slot, kc, vc, out=o_enc)
+        rc.compact_routes(kc, vc, keep, res_off, res_slot, res_len, vis, PACKED, route_cu, route_idx, k_route, v_route)
+        rc.attend_prefill(cq, ck, cv, cu_q, q_pos0, req.max_q, k_route, v_route, route_cu, out=o_pre)
+
+    for _ in range(3):
+        layer()
+    torch.cuda.synchronize(dev)
+    rl = np.diff(route_cu.cpu().numpy().astype(np.int64)).reshape(req.n_requests, g)
+    tq = np.diff(req.cu_q).astype(np.int64)
+    lens = pool.lens.astype(np.int64)
+    f_enc = 4 * d * int((lens * (lens + 1) // 2).sum()) * sh.n_q_heads
+    f_pre = 4 * d * int(sum(sh.group_size * (tq[b] * rl[b, kg] + tq[b] * (tq[b] + 1) // 2)
+                            for b in range(req.n_requests) for kg in range(g)))
+    rc.kernel_timer(True)
+    for _ in range(iters):
+        layer()
+    torch.cuda.synchronize(dev)
+    kt = rc.kernel_times()
+    rc.kernel_timer(False)
+    if rc.poll_status() != 0:
+        raise SystemExit("device status after the config-3 side measurement")
+    ms_e, ms_p = kt["encode_attn"][0] / iters, kt["prefill_attn"][0] / iters
+    return {"workload": "64 resources U[150,1200] (%d tokens), 16 requests of 4-12 resources, %d query tokens" % (
+                pool.total_tokens, req.total_q),
+            "encode_attn": {"tflops": f_enc / (ms_e * 1e-3) / 1e12, "ms": ms_e, "frac_of_bf16_peak": f_enc / (ms_e * 1e-3) / 1e12 / peak_tf},
+            "prefill_attn": {"tflops": f_pre / (ms_p * 1e-3) / 1e12, "ms": ms_p, "frac_of_bf16_peak": f_pre / (ms_p * 1e-3) / 1e12 / peak_tf}}
+
+
 class E2EPipeline:
     """End-to-end steps with the copies overlapped: two sets of device buffers
     and three streams, so that the copy-in of step k+1 and the copy-out of step
@@ -400,6 +455,7 @@ def main():
                     help="full = the benchmark workload; medium / small = reduced cases for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other", action="store_true", help="skip the side measurement of the composition-reuse shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -501,6 +557,10 @@ def main():
         stages["rope_store"] = {"gbs": w.bytes["rope_store"] / (t * 1e-3) / 1e9, "ms": t,
                                 "frac_of_hbm_peak": w.bytes["rope_store"] / (t * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
+    other = None
+    if rank == 0 and world == 1 and args.case == "full" and not args.no_other:
+        other = {"config3_layer": other_workload_config3(local, peak_tf)}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         f, sec, what = oracle_sample(w)
@@ -517,7 +577,7 @@ def main():
                            "useful_tflop_per_step": w.total_flops / 1e12,
                            "flops": {k: v / 1e12 for k, v in w.flops.items()}},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-                "cpu_baseline": cpu, "stages": stages, "kernels": per}
+                "cpu_baseline": cpu, "stages": stages, "kernels": per, "other_workloads": other}
         print(json.dumps(line))
     if dist:
         td.destroy_process_group()
