@@ -1,8 +1,7 @@
 // Tensor-core attention for encode and prefill (bf16, head_dim 128, Hq/G in {2,4,8}).
 //
 // Persistent kernel, one CTA per SM; a work item = (sequence, KV group, pair of
-// query tiles).  A
-// query tile is 128 rows = (128 / s) consecutive tokens x the s query heads of
+// query tiles).  A query tile is 128 rows = (128 / s) consecutive tokens x the s query heads of
 // the group, so every K/V tile is shared by all heads of the group and the
 // causal granularity is 128 / s tokens.  The two tiles of a CTA are consecutive
 // and share each K/V tile, read once from L2/HBM by TMA.
@@ -13,7 +12,9 @@
 //                them through a two-slot ring in shared memory
 //   warp  11     idle (completes the third warpgroup)
 //   warps 12-15  epilogue: O of a finished tile goes from tensor memory to HBM
-//                while the softmax warps already rotate the next item's Q
+//                while the softmax warps already rotate the next item's Q; in
+//                gather mode (route rows read from the resource cache through an
+//                index list) the same 128 lanes also fill the route's K/V tiles
 // setmaxnreg moves registers from warps 8-15 to the two softmax warpgroups,
 // which hold 128 scores per thread.
 //
@@ -21,8 +22,9 @@
 // S = Q K^T (both operands in 128B-swizzled shared memory, K-major); the softmax
 // warps read S with tcgen05.ld, keep a running maximum with lazy rescaling of O,
 // and write P = exp2(.) as bf16 over the first 64 columns of S; O += P V takes P
-// from tensor memory and V (MN-major) from shared memory.  While one tile's
-// softmax runs, the tensor core works on the other tile.
+// from tensor memory and V (MN-major) from shared memory, the first 64 keys as
+// soon as their half of P is stored.  While one tile's softmax runs, the tensor
+// core works on the other tile.
 //
 // Key tiles of an item: first the route's packed rows (all visible), then the
 // causal rows of the sequence itself up to the tile pair's last token.  The
