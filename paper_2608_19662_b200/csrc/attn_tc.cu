@@ -236,6 +236,17 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
       "mov.b64 {%0, %1}, rd;\n\t}"
       : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
+// d = a * b + c and d = a * b on pairs (one instruction each; same rounding as the scalar forms)
+__device__ __forceinline__ void fma2v(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void mul2v(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -813,10 +824,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           for (int i = 0; i < 4; ++i) {
             const float l0 = __uint_as_float(wlo[i] << 16), l1 = __uint_as_float(wlo[i] & 0xffff0000u);
             const float h0 = __uint_as_float(whi[i] << 16), h1 = __uint_as_float(whi[i] & 0xffff0000u);
-            ol[i] = pack2(__fmaf_rn(l0, cs[2 * i], -__fmul_rn(h0, sn[2 * i])),
-                          __fmaf_rn(l1, cs[2 * i + 1], -__fmul_rn(h1, sn[2 * i + 1])));
-            oh[i] = pack2(__fmaf_rn(h0, cs[2 * i], __fmul_rn(l0, sn[2 * i])),
-                          __fmaf_rn(h1, cs[2 * i + 1], __fmul_rn(l1, sn[2 * i + 1])));
+            // lo' = lo cos - hi sin, hi' = hi cos + lo sin: the products with sin are rounded first
+            // (hi * (-sin) is exactly -(hi * sin)), as in the scalar form of the other kernels
+            float t0, t1, u0, u1, a0, a1, b0, b1;
+            mul2v(t0, t1, h0, h1, -sn[2 * i], -sn[2 * i + 1]);
+            mul2v(u0, u1, l0, l1, sn[2 * i], sn[2 * i + 1]);
+            fma2v(a0, a1, l0, l1, cs[2 * i], cs[2 * i + 1], t0, t1);
+            fma2v(b0, b1, h0, h1, cs[2 * i], cs[2 * i + 1], u0, u1);
+            ol[i] = pack2(a0, a1);
+            oh[i] = pack2(b0, b1);
           }
           *reinterpret_cast<uint4*>(qb) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
           *reinterpret_cast<uint4*>(qb + BOX_BYTES) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
