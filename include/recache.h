@@ -110,7 +110,11 @@ RECACHE_API recache_status recache_poll_status(recache_ctx* ctx, void* stream, i
  * launch stream (a few microseconds of host time per launch).
  *   recache_kernel_count()      number of distinct kernels K
  *   recache_kernel_name(id)     static string, id in [0, K)
- *   recache_kernel_timer(ctx,e) enable (1) / disable (0); clears counters and pending events
+ *   recache_kernel_timer(ctx,e) 0 = off, 1 = every launch, 2 = the two attention launches only (light
+ *       enough to leave on inside a timed region); clears counters and pending events.
+ *       With 0 or 2 the small set-up kernel of the tensor-core attention runs on a
+ *       second stream of the context beside the call's first kernel (forked from and
+ *       joined to the caller's stream by events); with 1 everything stays on one stream.
  *   recache_kernel_times(ctx, ms_total[K], launches[K])  waits for the recorded
  *       events, returns per-kernel summed device time in ms (0 when the timer
  *       was off) and launch counts since the last clear, then clears both.

@@ -167,8 +167,9 @@ class ReCache:
         self._check(self.lib.recache_poll_status(self.h, _stream(), C.byref(code)), "recache_poll_status")
         return int(code.value)
 
-    def kernel_timer(self, enable: bool):
-        self._check(self.lib.recache_kernel_timer(self.h, 1 if enable else 0), "recache_kernel_timer")
+    def kernel_timer(self, enable):
+        """False / 0: off; True / 1: an event pair around every launch; 2: around the attention launches only."""
+        self._check(self.lib.recache_kernel_timer(self.h, int(enable)), "recache_kernel_timer")
 
     def kernel_times(self):
         """{kernel name: (total ms, launches)} since the last call; clears the counters."""

@@ -67,7 +67,10 @@ recache_status recache_create(recache_ctx** out, const recache_desc* desc, int d
             cudaMalloc(&ctx->status, 256) == cudaSuccess &&
             cudaMemcpy(ctx->cos_tab, c.data(), n * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
             cudaMemcpy(ctx->sin_tab, s.data(), n * sizeof(float), cudaMemcpyHostToDevice) == cudaSuccess &&
-            cudaMemset(ctx->status, 0, 256) == cudaSuccess;
+            cudaMemset(ctx->status, 0, 256) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     recache_destroy(ctx);
@@ -82,6 +85,9 @@ void recache_destroy(recache_ctx* ctx) {
   cudaFree(ctx->cos_tab);
   cudaFree(ctx->sin_tab);
   cudaFree(ctx->status);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->side) cudaStreamDestroy(ctx->side);
   clear_timer(ctx);
   delete ctx;
 }
@@ -110,6 +116,7 @@ recache_status recache_kernel_timer(recache_ctx* ctx, int32_t enable) {
   if (!ctx) return RECACHE_EINVAL;
   clear_timer(ctx);
   ctx->timer_on = enable != 0;
+  ctx->timer_attn_only = enable == 2;
   return RECACHE_OK;
 }
 
@@ -171,6 +178,7 @@ static recache_status encode_impl(recache_ctx* ctx, const void* q, const void* k
 
   RopeStoreArgs ra{k, v, k_cache, v_cache, cu_seqlens, n_resources, total_tokens, dst_slot, pos_offset,
                    pool_tokens, 0};
+  rc_fork_point(ctx, st);
   RC_CUDA(rc_launch_rope_store(ctx, ra, st), "encode: rope/store launch");
   EncodeArgs ea{q, out_o, out_dtype, cu_seqlens, n_resources, total_tokens, max_len, dst_slot,
                 k_cache, v_cache, pool_tokens, workspace, workspace_bytes, k_prefix, v_prefix, prefix_len, pos_offset};
@@ -261,6 +269,7 @@ static recache_status prefill_impl(recache_ctx* ctx, const void* q, const void* 
   RopeStoreArgs ra{k_conv, v_conv, k_conv_out, v_conv_out, cu_q, n_requests, total_q, conv_slot, q_pos0,
                    conv_rows, conv_slot ? 2 : 1};
   ra.hist = hist_len;
+  rc_fork_point(ctx, st);
   RC_CUDA(rc_launch_rope_store(ctx, ra, st), "prefill: rope/store launch");
   PrefillArgs pa{q, out_o, out_dtype, cu_q, q_pos0, n_requests, total_q, max_q, k_route, v_route, route_cu,
                  route_rows, k_conv_out, v_conv_out, workspace, workspace_bytes, conv_rows, conv_slot, hist_len};

@@ -1050,8 +1050,18 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
   p.gather_k = (const uint8_t*)a.k_cache; p.gather_v = (const uint8_t*)a.v_cache; p.route_idx = a.route_idx;
   p.pool_tokens = a.pool_tokens;
   {
-    RcLaunchScope scope(ctx, RC_K_TILE_PLAN, st);
-    tile_plan_kernel<<<1, 1024, 0, st>>>(p, tc_tok_per_cta(ctx), n_levels, items, level_off, order, (int)max_items);
+    // The work list only depends on the index arrays: when the caller marked a fork point before the
+    // rotate-and-store pass, it is built on the side stream beside that pass.
+    const bool fork = ctx->forked && cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess;
+    ctx->forked = false;
+    cudaStream_t ps = fork ? ctx->side : st;
+    {
+      RcLaunchScope scope(ctx, RC_K_TILE_PLAN, ps);
+      tile_plan_kernel<<<1, 1024, 0, ps>>>(p, tc_tok_per_cta(ctx), n_levels, items, level_off, order, (int)max_items);
+    }
+    if (fork && (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess ||
+                 cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess))
+      return cudaErrorUnknown;
   }
   const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
   const unsigned grid = (unsigned)(max_items * G < sms ? max_items * G : sms);

@@ -25,8 +25,15 @@ struct recache_ctx {
   int32_t* status;    // device status word
   int sm_count;
   std::string err;
+  // A second stream for small set-up kernels that do not depend on the call's first kernel (the work
+  // list of the tensor-core attention beside the rotate-and-store pass): forked from and joined to
+  // the caller's stream with the two events, so the caller sees one stream's ordering.
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  mutable bool forked = false;   // ev_fork was recorded for the call in progress
   // launch accounting (host side only)
   mutable bool timer_on = false;
+  mutable bool timer_attn_only = false;   // bracket the two attention launches only
   mutable int64_t launches[RC_K_COUNT] = {0};
   mutable std::vector<RcTimedLaunch> timed;
 };
@@ -37,7 +44,7 @@ struct RcLaunchScope {
   const recache_ctx* ctx; cudaStream_t st; cudaEvent_t stop = nullptr;
   RcLaunchScope(const recache_ctx* c, int id, cudaStream_t s) : ctx(c), st(s) {
     ctx->launches[id]++;
-    if (ctx->timer_on) {
+    if (ctx->timer_on && (!ctx->timer_attn_only || id == RC_K_ENCODE_ATTN || id == RC_K_PREFILL_ATTN)) {
       RcTimedLaunch t{id, nullptr, nullptr};
       if (cudaEventCreate(&t.start) == cudaSuccess && cudaEventCreate(&t.stop) == cudaSuccess) {
         cudaEventRecord(t.start, st);
@@ -48,6 +55,13 @@ struct RcLaunchScope {
   }
   ~RcLaunchScope() { if (stop) cudaEventRecord(stop, st); }
 };
+
+// Marks the point of the caller's stream that the side stream may start from (everything enqueued
+// before the call): record it before the call's first kernel.
+// (Not while the timer brackets every kernel: its event pairs are meant for kernels that run alone.)
+inline void rc_fork_point(const recache_ctx* ctx, cudaStream_t st) {
+  ctx->forked = ctx->side && (!ctx->timer_on || ctx->timer_attn_only) && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess;
+}
 
 // First device-side error wins.
 __device__ __forceinline__ void rc_set_status(int32_t* status, int32_t code) {
