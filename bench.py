@@ -45,7 +45,7 @@ from paper_2608_19662_b200 import workloads as wl  # noqa: E402
 # profiles/attn_tc_medium_case.md (dram__bytes_read.sum + dram__bytes_write.sum = 408.3 MB for 21,626
 # resource tokens).  The full workload is too large for a multi-pass capture; traffic grows in proportion
 # to the tokens (Q read, O written, K/V read once from HBM and re-read from L2), so it is scaled per token.
-NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 413.738e6 / 21626   # ncu: dram read + write of the 21,626-token encode launch (profiles/)
+NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 413.226e6 / 21626   # ncu: dram read + write of the 21,626-token encode launch (profiles/)
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -455,6 +455,9 @@ def main():
                     help="full = the benchmark workload; medium / small = reduced cases for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--timer-all", action="store_true",
+                    help="bracket every launch with events in the timed region too (keeps all kernels on one stream: "
+                         "the configuration the profiler captures were taken in)")
     ap.add_argument("--no-other", action="store_true", help="skip the side measurement of the composition-reuse shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -508,12 +511,12 @@ def main():
     # The timed region: event pairs around the two attention launches only (the roofline kernel's
     # duration comes from here).  A second, shorter pass brackets every launch for the per-kernel table;
     # that serialises the small set-up kernels and costs host time, so it is kept out of the value.
-    ms, kt_attn, clocks = timed(run.step, args.steps, with_timer=2, sample_clocks=True)
+    ms, kt_attn, clocks = timed(run.step, args.steps, with_timer=1 if args.timer_all else 2, sample_clocks=True)
     kt_steps = max(10, args.steps // 5) if not args.small else args.steps
     _, kt, _ = timed(run.step, kt_steps, with_timer=1)
     code = rc.poll_status()
     if code != 0:
-        raise SystemExit(f"device status {code} after the timed region")
+        raise SystemExit(f"device status {code} after the timed region ({rc.last_error()})")
     ms_step = ms / args.steps
     value = job_value(world, w.total_flops, ms_step)
 

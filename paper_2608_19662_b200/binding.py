@@ -167,6 +167,10 @@ class ReCache:
         self._check(self.lib.recache_poll_status(self.h, _stream(), C.byref(code)), "recache_poll_status")
         return int(code.value)
 
+    def last_error(self) -> str:
+        """Text of the context's last error (after a device time-out: which wait ran out)."""
+        return self.lib.recache_last_error(self.h).decode()
+
     def kernel_timer(self, enable):
         """False / 0: off; True / 1: an event pair around every launch; 2: around the attention launches only."""
         self._check(self.lib.recache_kernel_timer(self.h, int(enable)), "recache_kernel_timer")

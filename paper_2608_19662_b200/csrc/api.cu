@@ -97,11 +97,19 @@ const char* recache_last_error(const recache_ctx* ctx) { return ctx ? ctx->err.c
 recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* device_code) {
   if (!ctx || !device_code) return RECACHE_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
-  int32_t code = 0;
-  RC_CUDA(cudaMemcpyAsync(&code, ctx->status, sizeof(code), cudaMemcpyDeviceToHost, st), "poll copy");
-  RC_CUDA(cudaMemsetAsync(ctx->status, 0, sizeof(int32_t), st), "poll clear");
+  int32_t code[2] = {0, 0};   // the code, and where a wait ran out
+  RC_CUDA(cudaMemcpyAsync(code, ctx->status, sizeof(code), cudaMemcpyDeviceToHost, st), "poll copy");
+  RC_CUDA(cudaMemsetAsync(ctx->status, 0, sizeof(code), st), "poll clear");
   RC_CUDA(cudaStreamSynchronize(st), "poll sync");
-  *device_code = code;
+  *device_code = code[0];
+  if (code[0] == RECACHE_DEV_TIMEOUT) {
+    const uint32_t w = (uint32_t)code[1];
+    char msg[160];
+    snprintf(msg, sizeof(msg), "a kernel gave up waiting: %s, block %u, barrier slot %u, warp %u",
+             (w >> 28) == 1 ? "tensor-core attention" : (w >> 28) == 2 ? "split-KV decode" : "?", (w >> 16) & 0xfffu,
+             (w >> 8) & 0xffu, w & 0xffu);
+    ctx->err = msg;
+  }
   return RECACHE_OK;
 }
 

@@ -94,7 +94,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return;
     if ((it & 63) == 63) {
       if (*abort_flag) return;
-      if (clock64() - t0 > WAIT_CYCLES) { *abort_flag = 1; rc_set_status(status, RECACHE_DEV_TIMEOUT); return; }
+      if (clock64() - t0 > WAIT_CYCLES) { *abort_flag = 1; rc_set_timeout(status, RC_WHERE_DECODE_SPLIT, bar); return; }
     }
   }
 }
