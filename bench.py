@@ -259,6 +259,56 @@ def other_workload_config3(device: int, peak_tf: float, iters: int = 20):
             "prefill_attn": {"tflops": f_pre / (ms_p * 1e-3) / 1e12, "ms": ms_p, "frac_of_bf16_peak": f_pre / (ms_p * 1e-3) / 1e12 / peak_tf}}
 
 
+def other_workload_config5_dense(device: int, peak_tf: float, pool, req, iters: int = 10):
+    """The dense comparison point of the long-tool-set shape: the same 2048-token prefill with every route
+    seeing every token of all 64 resources (keep-all masks, all-visible routes), over a resident cache.
+    Attention throughput of the prefill launch from the library's event timer; compaction time beside it.
+    A side measurement: not part of `value`."""
+    from paper_2608_19662_b200 import PACKED, ReCache
+    pool, req = wl.keep_all(pool), wl.all_visible(req)   # the benchmark's own pool and request, masks and routes opened
+    sh = pool.shape
+    dev = torch.device("cuda", device)
+    g, d = sh.n_kv_heads, sh.head_dim
+    max_pos = int(req.q_pos0.max() + req.max_q) + 1
+    rc = ReCache(sh.n_q_heads, g, d, sh.rope_theta, sh.dtype, max_pos=max_pos, page_tokens=wl.PAGE_TOKENS, device=device)
+    t = lambda a: (torch.from_numpy(np.ascontiguousarray(a)) if isinstance(a, np.ndarray) else a).to(dev)
+    keep, res_off, res_slot, res_len, vis = t(pool.keep), t(req.res_off), t(req.res_slot), t(req.res_len), t(req.vis)
+    cq, ck, cv, cu_q, q_pos0 = t(req.q), t(req.k_conv), t(req.v_conv), t(req.cu_q), t(req.q_pos0)
+    kc = wl.seeded_normal(91, (g, pool.pool_tokens, d), sh.torch_dtype, device=dev)   # stand-in for an earlier encode
+    vc = wl.seeded_normal(92, (g, pool.pool_tokens, d), sh.torch_dtype, device=dev)
+    n_routes = req.n_requests * g
+    cap = int(req.res_len.sum()) * g + 64
+    route_cu = torch.empty(n_routes + 1, dtype=torch.int32, device=dev)
+    route_idx = torch.empty(cap, dtype=torch.int32, device=dev)
+    k_route, v_route = torch.empty((cap, d), dtype=sh.torch_dtype, device=dev), torch.empty((cap, d), dtype=sh.torch_dtype, device=dev)
+    o_pre = torch.empty((req.total_q, sh.n_q_heads, d), dtype=sh.torch_dtype, device=dev)
+
+    def layer():
+        rc.compact_routes(kc, vc, keep, res_off, res_slot, res_len, vis, PACKED, route_cu, route_idx, k_route, v_route)
+        rc.attend_prefill(cq, ck, cv, cu_q, q_pos0, req.max_q, k_route, v_route, route_cu, out=o_pre)
+
+    for _ in range(3):
+        layer()
+    torch.cuda.synchronize(dev)
+    rl = np.diff(route_cu.cpu().numpy().astype(np.int64)).reshape(req.n_requests, g)
+    tq = np.diff(req.cu_q).astype(np.int64)
+    f_pre = 4 * d * int(sum(sh.group_size * (tq[b] * rl[b, kg] + tq[b] * (tq[b] + 1) // 2)
+                            for b in range(req.n_requests) for kg in range(g)))
+    rc.kernel_timer(True)
+    for _ in range(iters):
+        layer()
+    torch.cuda.synchronize(dev)
+    kt = rc.kernel_times()
+    rc.kernel_timer(False)
+    if rc.poll_status() != 0:
+        raise SystemExit("device status after the config-5 dense side measurement")
+    ms_p, ms_g = kt["prefill_attn"][0] / iters, kt["compact_gather"][0] / iters
+    gather_bytes = int(rl.sum()) * d * 2 * 2 * 2          # K and V rows read and written
+    return {"workload": "2048 query tokens over all %d resource tokens per group (keep-all, all routes visible)" % int(rl[0, 0]),
+            "prefill_attn": {"tflops": f_pre / (ms_p * 1e-3) / 1e12, "ms": ms_p, "frac_of_bf16_peak": f_pre / (ms_p * 1e-3) / 1e12 / peak_tf},
+            "compact_gather": {"gbs": gather_bytes / (ms_g * 1e-3) / 1e9, "ms": ms_g}}
+
+
 class E2EPipeline:
     """End-to-end steps with the copies overlapped: two sets of device buffers
     and three streams, so that the copy-in of step k+1 and the copy-out of step
@@ -570,7 +620,8 @@ def main():
 
     other = None
     if rank == 0 and world == 1 and args.case == "full" and not args.no_other:
-        other = {"config3_layer": other_workload_config3(local, peak_tf)}
+        other = {"config3_layer": other_workload_config3(local, peak_tf),
+                 "config5_dense_prefill": other_workload_config5_dense(local, peak_tf, w.pool, w.req)}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
