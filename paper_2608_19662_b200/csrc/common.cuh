@@ -67,9 +67,9 @@ inline void rc_fork_point(const recache_ctx* ctx, cudaStream_t st) {
 __device__ __forceinline__ void rc_set_status(int32_t* status, int32_t code) {
   atomicCAS(status, 0, code);
 }
-// A bounded wait that ran out also says where (second status word, first one wins):
+// A bounded wait of the split-KV decode kernel that ran out also says where (second status word, first one wins):
 // kernel tag << 28 | (block & 0xfff) << 16 | (barrier's shared address / 8 & 0xff) << 8 | warp.
-constexpr uint32_t RC_WHERE_ATTN_TC = 1, RC_WHERE_DECODE_SPLIT = 2;
+constexpr uint32_t RC_WHERE_DECODE_SPLIT = 2;
 __device__ __forceinline__ void rc_set_timeout(int32_t* status, uint32_t kernel_tag, uint32_t bar) {
   atomicCAS(status, 0, (int32_t)RECACHE_DEV_TIMEOUT);
   const uint32_t where = kernel_tag << 28 | (blockIdx.x & 0xfffu) << 16 | ((bar >> 3) & 0xffu) << 8 | (threadIdx.x >> 5);
