@@ -68,7 +68,7 @@ constexpr uint32_t COL_S = 0, COL_O = 256;           // + 128 * tile
 
 constexpr int SORT_MAX = 4096;                      // work items up to which the plan sorts a prefill by weight (encode: a quarter)
 
-constexpr long long WAIT_CYCLES = 4000000000ll;      // ~2 s: a wait this long is a bug, not load
+constexpr uint32_t WAIT_PROBES = 1u << 21;           // ~2.8 s of suspended probes: a wait this long is a bug, not load
 
 struct TcParams {
   const int2* items; int32_t* header;   // header[0] = number of items, header[1] = work counter, header[2] = order[] is valid
@@ -103,19 +103,21 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after WAIT_CYCLES (or as soon as another thread of the
-// CTA has given up), records the failure in the device status word and lets the
-// kernel run to its end so that tensor memory is released.
+// Bounded wait: gives up after WAIT_PROBES unsuccessful probes (or as soon as another thread of
+// the CTA has given up), records the failure in the device status word and lets the kernel run to
+// its end so that tensor memory is released.  The bound is a probe count, not a clock reading:
+// a probe that fails has suspended the thread for about 1.3 us (measured), and the loop then
+// holds no 64-bit start time across it: the 32-register warps of this kernel are sensitive to
+// every register and instruction around their waits.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
   if (mbar_try(bar, parity)) return;
-  const long long t0 = clock64();
-  for (uint32_t it = 0;; ++it) {
+  for (uint32_t it = 1;; ++it) {
     if (mbar_try(bar, parity)) return;
-    if ((it & 63) == 63) {
+    if ((it & 1023u) == 0u) {
       if (*abort_flag) return;
-      if (clock64() - t0 > WAIT_CYCLES) {
+      if (it >= WAIT_PROBES) {   // (no location word here: even one more instruction on this cold path costs the kernel 6 %)
         *abort_flag = 1;
-        rc_set_status(status, RECACHE_DEV_TIMEOUT);   // (no location word here: even one more instruction on this cold path costs the kernel 6 %)
+        rc_set_status(status, RECACHE_DEV_TIMEOUT);
         return;
       }
     }
@@ -456,7 +458,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
   auto fetch_item = [&](uint32_t n, Item& it, bool release) {
     const int sl = n & 1u;
     mbar_wait(bar(B_IFULL + sl), (n >> 1) & 1u, abort_flag, p.status);
-    const volatile int* r = item_ring + sl * IT_WORDS;
+    const int* r = const_cast<const int*>(item_ring) + sl * IT_WORDS;   // (ordered by the barrier wait above and the arrive below)
     it.n_tiles = r[IT_NTILES]; it.g = r[IT_G]; it.seq0 = r[IT_SEQ0]; it.L = r[IT_L]; it.tok0 = r[IT_TOK0];
     it.kv_end = r[IT_KVEND]; it.pos0 = r[IT_POS0]; it.rA0 = r[IT_RA0]; it.lenA = r[IT_LENA]; it.nA = r[IT_NA];
     it.b_valid = r[IT_BVALID]; it.H = r[IT_H];
