@@ -943,6 +943,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
   }
   // ---- teardown: every thread is done with tensor memory before it is freed ----
+  if (*abort_flag) {
+    // A wait ran out: the roles fell through their loops with loads, copies and MMAs possibly still in
+    // flight.  Let them land (none depends on another CTA; ~100 us is far more than any of them takes)
+    // before shared and tensor memory go away under them.
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000ll) { }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 9) {

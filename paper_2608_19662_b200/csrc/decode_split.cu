@@ -412,6 +412,13 @@ __global__ void __launch_bounds__(GATHER ? NTHREADS_GATHER : NTHREADS, 1) decode
       bar_consumers();
     }
   }
+  if (*abort_flag) {
+    // A wait ran out: loads may still be in flight towards this CTA's shared memory.  Let them
+    // land (~100 us is far more than any of them takes) before the CTA ends.
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    const long long t0 = clock64();
+    while (clock64() - t0 < 200000ll) { }
+  }
 }
 
 // Combines the splits of every (sequence, head): grid = batch * Hq, 32 threads x 4 dims.
