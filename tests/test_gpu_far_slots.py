@@ -90,3 +90,28 @@ def test_pages_past_two_to_the_31_elements():
                             storage=sh.dtype)
     assert max_abs(od, ref) < 1e-2
     assert rc.poll_status() == 0
+
+
+def test_positions_near_the_end_of_a_long_rotary_table():
+    """A conversation that starts at position 130,000 of a 131,072-row cos/sin table (angles of up to 1.3e5
+    radians for the fastest frequency: the table is built in double precision on the host); the last query
+    token sits on the table's last row."""
+    sh = wl.QWEN3_4B
+    g = sh.n_kv_heads
+    max_pos = 131072
+    rng = np.random.default_rng(5)
+    lens = [200, 90]
+    pool = wl.pack_resources(sh, 55, lens, wl.keep_mask_spans(rng, lens))
+    vis = wl.routes_random(rng, g, 2, 0.5)
+    tq = 300
+    req = wl.make_requests(sh, 56, pool, [[0, 1]], [vis], [tq], q_pos0=[max_pos - tq])
+    rc = make_ctx(sh, max_pos=max_pos)
+    _, kc_ref, vc_ref = oracle_encode(pool)
+    _, kc, vc = gpu_encode(rc, pool)
+    out = gpu_compact(rc, pool, req, kc, vc)
+    p, k_hat, _ = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
+    p_ref, k_hat_ref = oracle_prefill(req, oracle_rows(pool, req), kc_ref, vc_ref)
+    assert max_abs(p, p_ref) < 1e-2
+    # rotated conversation keys at these positions: one bf16 ulp at most (values up to ~4: ulp 2^-6)
+    assert max_abs(k_hat.transpose(0, 1) if k_hat.shape[0] == g else k_hat, k_hat_ref) <= 2.0 ** -6
+    assert rc.poll_status() == 0
