@@ -309,6 +309,51 @@ def other_workload_config5_dense(device: int, peak_tf: float, pool, req, iters: 
             "compact_gather": {"gbs": gather_bytes / (ms_g * 1e-3) / 1e9, "ms": ms_g}}
 
 
+def other_workload_config4_shared_pool(device: int, hbm_gbs: float, iters: int = 20):
+    """Decode of the 64-sequence batch when every sequence routes to the SAME 16 resources: the resource pages of
+    a KV group are shared by all sequences (one page table row copied to the whole batch), the 2048-row
+    histories stay private.  Logical bytes per step are those of the primary case; the shared pages are read
+    from HBM once and from L2 after that.  The primary case (every item its own pages) is timed beside it on
+    the same page pool.  A side measurement: not part of `value`."""
+    from paper_2608_19662_b200 import ReCache
+    dec = wl.config4_decode()
+    sh = dec.shape
+    dev = torch.device("cuda", device)
+    g, d = sh.n_kv_heads, sh.head_dim
+    rc = ReCache(sh.n_q_heads, g, d, sh.rope_theta, sh.dtype, max_pos=int(dec.q_pos.max()) + 2, page_tokens=wl.PAGE_TOKENS,
+                 device=device)
+    t = lambda a: (torch.from_numpy(np.ascontiguousarray(a)) if isinstance(a, np.ndarray) else a).to(dev)
+    q, q_pos, kp, vp = t(dec.q), t(dec.q_pos), t(dec.k_pages), t(dec.v_pages)
+    hpt, hlen = t(dec.hist_page_table), t(dec.hist_len)
+    batch = dec.q.shape[0]
+    shared_pt = np.tile(dec.res_page_table[:g], (batch, 1))
+    shared_len = np.tile(dec.res_len[:g], batch)
+    out = torch.empty((batch, sh.n_q_heads, d), dtype=sh.torch_dtype, device=dev)
+    res = {}
+    for name, rpt, rlen in (("private_pages", dec.res_page_table, dec.res_len), ("shared_pool", shared_pt, shared_len)):
+        d_rpt, d_rlen = t(rpt), t(rlen)
+        run = lambda: rc.attend_decode(q, q_pos, kp, vp, d_rpt, d_rlen, hpt, hlen, out=out)
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize(dev)
+        rc.kernel_timer(True)
+        for _ in range(iters):
+            run()
+        torch.cuda.synchronize(dev)
+        kt = rc.kernel_times()
+        rc.kernel_timer(False)
+        ms = (kt["decode_attn"][0] + kt["decode_merge"][0]) / iters
+        logical = int((rlen.astype(np.int64) + dec.hist_len.astype(np.int64)).sum()) * d * 2 * 2
+        unique_pages = len(np.unique(np.concatenate([rpt[rpt >= 0].ravel(), dec.hist_page_table[dec.hist_page_table >= 0].ravel()])))
+        res[name] = {"ms": ms, "logical_gbs": logical / (ms * 1e-3) / 1e9, "logical_bytes": logical,
+                     "unique_page_bytes": unique_pages * wl.PAGE_TOKENS * d * 2 * 2,
+                     "logical_frac_of_hbm_peak": logical / (ms * 1e-3) / 1e9 / hbm_gbs}
+    if rc.poll_status() != 0:
+        raise SystemExit("device status after the shared-pool decode side measurement")
+    res["workload"] = "decode batch 64, 4 of 16 resources per route (~600 tokens, 30% kept), 2048-row private histories"
+    return res
+
+
 class E2EPipeline:
     """End-to-end steps with the copies overlapped: two sets of device buffers
     and three streams, so that the copy-in of step k+1 and the copy-out of step
@@ -621,7 +666,8 @@ def main():
     other = None
     if rank == 0 and world == 1 and args.case == "full" and not args.no_other:
         other = {"config3_layer": other_workload_config3(local, peak_tf),
-                 "config5_dense_prefill": other_workload_config5_dense(local, peak_tf, w.pool, w.req)}
+                 "config5_dense_prefill": other_workload_config5_dense(local, peak_tf, w.pool, w.req),
+                 "config4_decode_shared_pool": other_workload_config4_shared_pool(local, peaks["hbm_gbs"])}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
