@@ -82,3 +82,36 @@ def test_random_case(seed):
                                storage="bf16", hist_k=hk, hist_v=hv)
     assert max_abs(od, rd) < 1e-2
     assert rc.poll_status() == 0
+
+
+@pytest.mark.parametrize("seed", list(range(6)))
+def test_random_multi_tile_case(seed):
+    """The same idea at sizes that span many K/V tiles: resources of up to 1600 tokens, up to 700 query
+    tokens per request, 2 / 4 / 8 query heads per KV group, span-shaped keep masks, gaps between cache slots;
+    encode, compaction, packed prefill and the zero-copy prefill (which must agree bit for bit)."""
+    from pipeline import gpu_prefill, oracle_prefill
+    rng = np.random.default_rng(7000 + seed)
+    sh = [wl.QWEN3_4B, wl.Shape(16, 8, 128, 1e6, "bf16"), wl.Shape(16, 2, 128, 1e4, "bf16")][seed % 3]
+    g = sh.n_kv_heads
+    n_res = int(rng.integers(2, 6))
+    lens = [int(x) for x in rng.integers(100, 1600, n_res)]
+    pool = wl.pack_resources(sh, 8000 + seed, lens, wl.keep_mask_spans(rng, lens), slot_gap=int(rng.integers(0, 70)))
+    B = int(rng.integers(1, 4))
+    res_lists = [[int(x) for x in rng.permutation(n_res)[:int(rng.integers(1, n_res + 1))]] for _ in range(B)]
+    vis = [(rng.random((g, len(l))) < 0.6).astype(np.uint8) for l in res_lists]
+    tq = [int(x) for x in rng.integers(1, 700, B)]
+    rc = make_ctx(sh, max_pos=16384)
+    o_ref, kc_ref, vc_ref = oracle_encode(pool)
+    o, kc, vc = gpu_encode(rc, pool)
+    assert max_abs(o, o_ref) < 1e-2
+    req = wl.make_requests(sh, 9000 + seed, pool, res_lists, vis, tq)
+    rows = oracle_rows(pool, req)
+    out = gpu_compact(rc, pool, req, kc, vc)
+    assert np.array_equal(out["route_cu"].cpu().numpy(), orc.route_prefix(rows))
+    p, _, _ = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
+    p_ref, _ = oracle_prefill(req, rows, kc_ref, vc_ref)
+    assert max_abs(p, p_ref) < 1e-2
+    p_g, _, _ = rc.attend_prefill_gather(dev(req.q), dev(req.k_conv), dev(req.v_conv), dev(req.cu_q), dev(req.q_pos0),
+                                         req.max_q, kc, vc, out["route_idx"], out["route_cu"], out_dtype=torch.float32)
+    assert torch.equal(p_g, p)
+    assert rc.poll_status() == 0
