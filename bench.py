@@ -45,7 +45,7 @@ from paper_2608_19662_b200 import workloads as wl  # noqa: E402
 # profiles/attn_tc_medium_case.md (dram__bytes_read.sum + dram__bytes_write.sum = 408.3 MB for 21,626
 # resource tokens).  The full workload is too large for a multi-pass capture; traffic grows in proportion
 # to the tokens (Q read, O written, K/V read once from HBM and re-read from L2), so it is scaled per token.
-NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 414.329e6 / 21626   # ncu: dram read + write of the 21,626-token encode launch (profiles/)
+NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 413.339e6 / 21626   # ncu: dram read + write of the 21,626-token encode launch (profiles/)
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
