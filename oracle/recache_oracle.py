@@ -26,6 +26,10 @@ order then ascending token; rotated queries and keys are materialised in the
 storage dtype (`storage`: "bf16", "f32" or None = keep fp64) before the score
 product, as a transformer running in that dtype does, so the key a resource's
 own tokens attend to is the very key the cache holds for every later reader.
+Rounding the rotated KEY is forced by the method (a cached block is reused as
+stored); rounding the rotated QUERY is a reading, and `round_q=False` evaluates
+the other one (query kept in fp64 after the rotation) so that the tests can say
+what the reading is worth.
 
 Pins (tests/test_oracle_*.py): hand-computed RoPE values, brute-force masked
 attention in pure Python, torch's fp64 scaled_dot_product_attention on the
@@ -89,7 +93,8 @@ def _softmax_rows(s: np.ndarray) -> np.ndarray:
 
 # ----------------------------------------------------------------- encode --
 def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] = None,
-                     pos_offset: Optional[Sequence[int]] = None, prefix_k=None, prefix_v=None):
+                     pos_offset: Optional[Sequence[int]] = None, prefix_k=None, prefix_v=None,
+                     round_q: bool = True):
     """Resource-wise encoding.  q: [T,Hq,d]; k, v: [T,G,d] (pre-RoPE), resource
     i = rows cu_seqlens[i]..cu_seqlens[i+1]-1 at positions pos_offset[i] + 0..D_i-1
     (pos_offset = None: resource-local positions from 0; one common offset P: the
@@ -97,8 +102,8 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
     variant, which drops cross-resource attention but keeps original positions).
     prefix_k / prefix_v [G][P][d]: rotated keys / values of a shared prefix as a
     cache holds them; every resource token sees all of them besides its own
-    resource's tokens j' <= j ("attend only to the shared prefix and their local
-    resource tokens").
+    resource's tokens j' <= j (the shared-prefix form of resource-wise attention,
+    Section "Resource-Wise Attention").
     Returns (o [T,Hq,d], k_hat [T,G,d] in storage precision, v [T,G,d])."""
     q = np.asarray(q, F64); k = np.asarray(k, F64); v = np.asarray(v, F64)
     t, hq, d = q.shape
@@ -112,7 +117,7 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
         if n == 0:
             continue
         pos = np.arange(n) + (0 if pos_offset is None else int(pos_offset[i]))
-        qh = round_storage(rope(q[a:b], pos, theta), storage)
+        qh = round_storage(rope(q[a:b], pos, theta), storage if round_q else None)
         kh = round_storage(rope(k[a:b], pos, theta), storage)
         k_hat[a:b] = kh
         causal = np.tril(np.ones((n, n), dtype=bool))
@@ -130,7 +135,7 @@ def encode_resources(q, k, v, cu_seqlens, theta: float, storage: Optional[str] =
 
 
 def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int]],
-                storage: Optional[str] = None):
+                storage: Optional[str] = None, round_q: bool = True):
     """The same definition for a chosen set of output rows (token, head) only,
     one at a time; for sizes where the full table takes minutes.  q/k/v may be
     fp32 arrays holding bf16 values: only the rows a sample needs are widened."""
@@ -144,7 +149,8 @@ def encode_rows(q, k, v, cu_seqlens, theta: float, rows: Sequence[Tuple[int, int
         a = int(cu[i])
         j = tok - a
         kg = h // s
-        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([j]), theta), storage)[0, 0]
+        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([j]), theta),
+                           storage if round_q else None)[0, 0]
         kh = round_storage(rope(np.asarray(k[a:tok + 1, kg:kg + 1], F64), np.arange(j + 1), theta), storage)[:, 0, :]
         sc = kh @ qh / math.sqrt(d)
         out[n] = _softmax_rows(sc[None, :])[0] @ np.asarray(v[a:tok + 1, kg, :], F64)
@@ -227,7 +233,7 @@ def gather_paged(cache, rows, page_table, n_pages: int, page_tokens: int, fill=0
 
 # ------------------------------------------------------- routed attention --
 def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta: float,
-                   storage: Optional[str] = None, hist_k=None, hist_v=None):
+                   storage: Optional[str] = None, hist_k=None, hist_v=None, round_q: bool = True):
     """Conversation tokens of request b (positions q_pos0[b] + t) attend, in one
     softmax with scale 1/sqrt(d), to (i) every row of their route's compacted
     resource KV (cached rotated keys used as stored) and (ii) conversation
@@ -247,7 +253,7 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
         if n == 0:
             continue
         pos = int(q_pos0[b]) + np.arange(n)
-        qh = round_storage(rope(q[a:e], pos, theta), storage)
+        qh = round_storage(rope(q[a:e], pos, theta), storage if round_q else None)
         kh = round_storage(rope(k_conv[a:e], pos, theta), storage)
         kc_hat[a:e] = kh
         causal = np.tril(np.ones((n, n), dtype=bool))
@@ -267,7 +273,7 @@ def attend_prefill(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, thet
 
 
 def prefill_rows(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta: float,
-                 out_rows: Sequence[Tuple[int, int]], storage: Optional[str] = None):
+                 out_rows: Sequence[Tuple[int, int]], storage: Optional[str] = None, round_q: bool = True):
     """attend_prefill for chosen (query token, head) rows only."""
     cu = np.asarray(cu_q)
     tq, hq, d = q.shape
@@ -280,7 +286,8 @@ def prefill_rows(q, k_conv, v_conv, cu_q, q_pos0, rows, k_cache, v_cache, theta:
         t = tok - a
         kg = h // s
         p0 = int(q_pos0[b])
-        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([p0 + t]), theta), storage)[0, 0]
+        qh = round_storage(rope(np.asarray(q[tok:tok + 1, h:h + 1], F64), np.array([p0 + t]), theta),
+                           storage if round_q else None)[0, 0]
         kh = round_storage(rope(np.asarray(k_conv[a:tok + 1, kg:kg + 1], F64), p0 + np.arange(t + 1), theta),
                            storage)[:, 0, :]
         r = rows[b][kg]
@@ -308,7 +315,7 @@ def append_decode_kv(k_pages, v_pages, hist_page_table, hist_len, k_new, v_new, 
 
 def attend_decode(q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page_table,
                   hist_len, theta: float, page_tokens: int, items: Optional[Sequence[int]] = None,
-                  storage: Optional[str] = None):
+                  storage: Optional[str] = None, round_q: bool = True):
     """One query token per sequence over its route's paged resource rows and its
     paged history (whose last row is the current token).  q: [B,Hq,d] pre-RoPE.
     `items` restricts the work to chosen (sequence*G + group) items; other
@@ -317,7 +324,7 @@ def attend_decode(q, q_pos, k_pages, v_pages, res_page_table, res_len, hist_page
     b, hq, d = q.shape
     g = len(res_len) // b
     s = hq // g
-    qh = round_storage(rope(q, np.asarray(q_pos), theta), storage)
+    qh = round_storage(rope(q, np.asarray(q_pos), theta), storage if round_q else None)
     o = np.zeros_like(q)
 
     def rows_of(table, n):

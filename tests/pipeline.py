@@ -81,10 +81,10 @@ def gpu_prefill(rc, req, k_route, v_route, route_cu, out_dtype=torch.float32):
 
 
 # --------------------------------------------------------------- oracle side --
-def oracle_encode(pool: wl.ResourceBatch):
+def oracle_encode(pool: wl.ResourceBatch, round_q: bool = True):
     sh = pool.shape
     o, k_hat, v = orc.encode_resources(f64(pool.q), f64(pool.k), f64(pool.v), pool.cu_seqlens, sh.rope_theta,
-                                       storage=sh.dtype)
+                                       storage=sh.dtype, round_q=round_q)
     kc = np.full((sh.n_kv_heads, pool.pool_tokens, sh.head_dim), np.nan)
     vc = np.full_like(kc, np.nan)
     orc.write_cache(kc, vc, k_hat, v, pool.cu_seqlens, pool.dst_slot)
@@ -111,13 +111,28 @@ def oracle_rows(pool, req):
     return orc.compact_routes(pool.keep, req.res_off, req.res_slot, req.res_len, req.vis)
 
 
-def oracle_prefill(req, rows, kc, vc):
+def oracle_prefill(req, rows, kc, vc, round_q: bool = True):
     sh = req.shape
     return orc.attend_prefill(f64(req.q), f64(req.k_conv), f64(req.v_conv), req.cu_q, req.q_pos0, rows, kc, vc,
-                              sh.rope_theta, storage=sh.dtype)
+                              sh.rope_theta, storage=sh.dtype, round_q=round_q)
 
 
 # ---------------------------------------------------------------- comparisons --
+def report_readings(case: str, stage: str, gated: float, unrounded: float):
+    """The parity gate compares with the oracle whose rotated query is rounded to
+    the storage dtype (what the kernels compute).  Beside it, the error against
+    the oracle that keeps the rotated query exact (cached keys as stored) is
+    printed, and appended to the file RECACHE_PARITY_REPORT names, so that the
+    share of the tolerance the reading consumes is on record per case."""
+    import os
+    line = f"{case:28s} {stage:8s} max|gpu-oracle| = {gated:.3e}   vs oracle with unrounded query = {unrounded:.3e}"
+    print(line)
+    path = os.environ.get("RECACHE_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
 def max_abs(a, b):
     a, b = f64(a), f64(b)
     return float(np.abs(a - b).max()) if a.size else 0.0

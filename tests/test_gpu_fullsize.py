@@ -16,7 +16,8 @@ sys.path.insert(0, ROOT)
 from oracle import recache_oracle as orc
 from paper_2608_19662_b200 import workloads as wl
 
-from pipeline import f64, gpu_compact, gpu_encode, gpu_prefill, make_ctx, oracle_cache_only, sample_rows
+from pipeline import (f64, gpu_compact, gpu_encode, gpu_prefill, make_ctx, oracle_cache_only, report_readings,
+                      sample_rows)
 from test_gpu_parity import assert_rotated_close
 
 pytestmark = pytest.mark.gpu
@@ -51,6 +52,10 @@ def test_bench_step_full_size():
     o = run.o_enc.cpu()
     got = np.stack([f64(o[t, h]) for t, h in rows])
     assert _close(got, ref)
+    ref_u = orc.encode_rows(f32(pool.q), f32(pool.k), f32(pool.v), pool.cu_seqlens, sh.rope_theta, rows[:64],
+                            storage="bf16", round_q=False)
+    report_readings("config5 full (bf16 out)", "encode", float(np.abs(got - ref).max()),
+                    float(np.abs(got[:64] - ref_u).max()))
 
     # ---- packed compaction: exact ----
     rt = orc.compact_routes(pool.keep, req.res_off, req.res_slot, req.res_len, req.vis)
@@ -69,7 +74,12 @@ def test_bench_step_full_size():
     pref = orc.prefill_rows(f32(req.q), f32(req.k_conv), f32(req.v_conv), req.cu_q, req.q_pos0, rt, kc_ref, vc_ref,
                             sh.rope_theta, prow, storage="bf16")
     op = run.o_pre.cpu()
-    assert _close(np.stack([f64(op[t, h]) for t, h in prow]), pref)
+    gotp = np.stack([f64(op[t, h]) for t, h in prow])
+    assert _close(gotp, pref)
+    pref_u = orc.prefill_rows(f32(req.q), f32(req.k_conv), f32(req.v_conv), req.cu_q, req.q_pos0, rt, kc_ref, vc_ref,
+                              sh.rope_theta, prow[:64], storage="bf16", round_q=False)
+    report_readings("config5 full (bf16 out)", "prefill", float(np.abs(gotp - pref).max()),
+                    float(np.abs(gotp[:64] - pref_u).max()))
 
     # ---- paged compaction for the decode batch: exact ----
     rows4 = orc.compact_routes(dc.keep, dc.res_off, dc.dst_slot, dc.lens, dc.vis)

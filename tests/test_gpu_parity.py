@@ -11,7 +11,7 @@ from oracle import recache_oracle as orc
 from paper_2608_19662_b200 import workloads as wl
 
 from pipeline import (bf16_ulp_distance, dev, f64, gpu_compact, gpu_encode, gpu_prefill, make_ctx, max_abs,
-                      oracle_cache_only, oracle_encode, oracle_prefill, oracle_rows, sample_rows)
+                      oracle_cache_only, oracle_encode, oracle_prefill, oracle_rows, report_readings, sample_rows)
 
 pytestmark = pytest.mark.gpu
 
@@ -80,6 +80,7 @@ def test_config1_fp32_whole_path():
     o_ref, kc_ref, vc_ref = oracle_encode(pool)
     o, kc, vc = gpu_encode(rc, pool)
     assert max_abs(o, o_ref) < TOL_F32
+    report_readings("config1 fp32", "encode", max_abs(o, o_ref), max_abs(o, oracle_encode(pool, round_q=False)[0]))
     check_cache(sh, kc, vc, kc_ref, vc_ref)
     # position 0 is the identity: the first cached key row of every resource is its input, bitwise
     for i, s0 in enumerate(pool.dst_slot):
@@ -93,6 +94,8 @@ def test_config1_fp32_whole_path():
     p_ref, kconv_ref = oracle_prefill(req, rows, kc_ref, vc_ref)
     p, kconv, vconv = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
     assert max_abs(p, p_ref) < TOL_F32
+    report_readings("config1 fp32", "prefill", max_abs(p, p_ref),
+                    max_abs(p, oracle_prefill(req, rows, kc_ref, vc_ref, round_q=False)[0]))
     assert_rotated_close(sh, kconv, np.transpose(kconv_ref, (1, 0, 2)))
     assert torch.equal(vconv.cpu(), req.v_conv.permute(1, 0, 2))
     assert_status_ok(rc)
@@ -163,6 +166,8 @@ def test_config2_bf16_whole_path(out_dtype):
     o, kc, vc = gpu_encode(rc, pool, out_dtype=out_dtype)
     slack = 0.0 if out_dtype == torch.float32 else 2.0 ** -8      # half a bf16 ulp of the reference
     assert (np.abs(f64(o) - o_ref) <= TOL_BF16 + slack * np.abs(o_ref)).all()
+    tag = "config2 bf16 out=" + ("f32" if out_dtype == torch.float32 else "bf16")
+    report_readings(tag, "encode", max_abs(o, o_ref), max_abs(o, oracle_encode(pool, round_q=False)[0]))
     check_cache(sh, kc, vc, kc_ref, vc_ref)
     rows = oracle_rows(pool, req)
     lens = [len(r) for r in rows[0]]
@@ -173,6 +178,8 @@ def test_config2_bf16_whole_path(out_dtype):
     p_ref, kconv_ref = oracle_prefill(req, rows, kc_ref, vc_ref)
     p, kconv, vconv = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"], out_dtype=out_dtype)
     assert (np.abs(f64(p) - p_ref) <= TOL_BF16 + slack * np.abs(p_ref)).all()
+    report_readings(tag, "prefill", max_abs(p, p_ref),
+                    max_abs(p, oracle_prefill(req, rows, kc_ref, vc_ref, round_q=False)[0]))
     assert_rotated_close(sh, kconv, np.transpose(kconv_ref, (1, 0, 2)))
     assert torch.equal(vconv.cpu(), req.v_conv.permute(1, 0, 2))
     assert_status_ok(rc)
@@ -212,6 +219,8 @@ def test_config3_reuse_bit_identical_kv_and_permutation_invariance():
         kc_ref, vc_ref = oracle_cache_only(pool)
         p_ref, _ = oracle_prefill(req, rows, kc_ref, vc_ref)
         assert max_abs(p, p_ref) < TOL_BF16
+        report_readings(f"config3 small layer {layer}", "prefill", max_abs(p, p_ref),
+                        max_abs(p, oracle_prefill(req, rows, kc_ref, vc_ref, round_q=False)[0]))
         # same requests with every resource list reversed (and the route table permuted with it)
         perm = np.concatenate([np.arange(req.res_off[b], req.res_off[b + 1])[::-1] for b in range(req.n_requests)])
         req_p = wl.RequestBatch(**{**req.__dict__})
@@ -236,6 +245,10 @@ def test_config4_decode_small_batch():
                             dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS,
                             storage=sh.dtype)
     assert max_abs(od, ref) < TOL_BF16
+    ref_u = orc.attend_decode(f64(dec.q), dec.q_pos, f64(dec.k_pages), f64(dec.v_pages), dec.res_page_table,
+                              dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS,
+                              storage=sh.dtype, round_q=False)
+    report_readings("config4 small", "decode", max_abs(od, ref), max_abs(od, ref_u))
     assert_status_ok(rc)
 
 
@@ -252,10 +265,17 @@ def test_config4_decode_full_size_sampled_items():
                             dec.res_page_table,
                             dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta, wl.PAGE_TOKENS, items=items,
                             storage=sh.dtype)
+    ref_u = orc.attend_decode(f64(dec.q), dec.q_pos, dec.k_pages.float().numpy(), dec.v_pages.float().numpy(),
+                              dec.res_page_table, dec.res_len, dec.hist_page_table, dec.hist_len, sh.rope_theta,
+                              wl.PAGE_TOKENS, items=items, storage=sh.dtype, round_q=False)
     g, s = sh.n_kv_heads, sh.group_size
+    worst = worst_u = 0.0
     for it in items:
         b, kg = divmod(it, g)
         assert max_abs(od[b, kg * s:(kg + 1) * s], ref[b, kg * s:(kg + 1) * s]) < TOL_BF16
+        worst = max(worst, max_abs(od[b, kg * s:(kg + 1) * s], ref[b, kg * s:(kg + 1) * s]))
+        worst_u = max(worst_u, max_abs(od[b, kg * s:(kg + 1) * s], ref_u[b, kg * s:(kg + 1) * s]))
+    report_readings("config4 full (32 items)", "decode", worst, worst_u)
     assert_status_ok(rc)
 
 
@@ -267,6 +287,7 @@ def test_config5_scaled_routed_and_dense_comparison():
     o_ref, kc_ref, vc_ref = oracle_encode(pool)
     o, kc, vc = gpu_encode(rc, pool)
     assert max_abs(o, o_ref) < TOL_BF16
+    report_readings("config5 scaled", "encode", max_abs(o, o_ref), max_abs(o, oracle_encode(pool, round_q=False)[0]))
     for pl, rq in ((pool, req), (wl.keep_all(pool), wl.all_visible(req))):
         rows = oracle_rows(pl, rq)
         out = gpu_compact(rc, pl, rq, kc, vc)
@@ -275,4 +296,6 @@ def test_config5_scaled_routed_and_dense_comparison():
         p_ref, _ = oracle_prefill(rq, rows, kc_ref, vc_ref)
         p, _, _ = gpu_prefill(rc, rq, out["k_out"], out["v_out"], out["route_cu"])
         assert max_abs(p, p_ref) < TOL_BF16
+        report_readings("config5 scaled " + ("routed" if pl is pool else "dense"), "prefill", max_abs(p, p_ref),
+                        max_abs(p, oracle_prefill(rq, rows, kc_ref, vc_ref, round_q=False)[0]))
     assert_status_ok(rc)
