@@ -105,6 +105,16 @@ RECACHE_API const char* recache_last_error(const recache_ctx* ctx);
  * (and, for the split-KV decode kernel, the block, barrier and warp that gave up first). */
 RECACHE_API recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* device_code);
 
+/* Self-test of the failure path (no paper counterpart).  Every barrier wait inside the TMA kernels
+ * is bounded: a wait that runs out sets RECACHE_DEV_TIMEOUT, releases the CTA's other waits, lets
+ * the copies in flight land and the kernel end normally.  This call enqueues one small CTA that
+ * runs exactly that code (the same wait and drain helpers, probe bound 2^10, about a millisecond)
+ * on a barrier nobody arrives at.  report: DEVICE pointer to two int32: [0] = 1 if the wait gave
+ * up, [1] = thousands of SM cycles it waited.  Afterwards recache_poll_status() returns
+ * RECACHE_DEV_TIMEOUT once and recache_last_error() names the self-test; the context stays usable.
+ * Nothing hangs or faults. */
+RECACHE_API recache_status recache_selftest_wait_timeout(recache_ctx* ctx, int32_t* report, void* stream);
+
 /*
  * Launch accounting.  The library counts every kernel it launches; with the
  * timer enabled it also records a CUDA event pair around each launch on the

@@ -37,6 +37,7 @@ SIGNATURES = {
     "recache_poll_status": (C.c_int, [_P, _P, C.POINTER(_I32)]),
     "recache_kernel_count": (_I32, []),
     "recache_kernel_name": (C.c_char_p, [_I32]),
+    "recache_selftest_wait_timeout": (C.c_int, [_P, _P, _P]),
     "recache_kernel_timer": (C.c_int, [_P, _I32]),
     "recache_kernel_times": (C.c_int, [_P, C.POINTER(C.c_float), C.POINTER(_I64)]),
     "recache_encode_workspace_bytes": (_I64, [_P, _I32, _I32, _I32]),
@@ -166,6 +167,15 @@ class ReCache:
         code = _I32(0)
         self._check(self.lib.recache_poll_status(self.h, _stream(), C.byref(code)), "recache_poll_status")
         return int(code.value)
+
+    def selftest_wait_timeout(self):
+        """Runs the bounded-wait self-test kernel (a wait on a barrier nobody arrives at); returns
+        (gave_up, kilo-cycles waited).  poll_status() afterwards reports the time-out once."""
+        report = torch.zeros(2, dtype=torch.int32, device=self.device)
+        self._check(self.lib.recache_selftest_wait_timeout(self.h, _ptr(report), _stream()),
+                    "recache_selftest_wait_timeout")
+        r = report.cpu().tolist()
+        return bool(r[0]), int(r[1])
 
     def last_error(self) -> str:
         """Text of the context's last error (after a device time-out: which wait ran out)."""

@@ -108,10 +108,19 @@ recache_status recache_poll_status(recache_ctx* ctx, void* stream, int32_t* devi
     if ((w >> 28) == 2)
       snprintf(msg, sizeof(msg), "a kernel gave up waiting: split-KV decode, block %u, barrier slot %u, warp %u", (w >> 16) & 0xfffu,
                (w >> 8) & 0xffu, w & 0xffu);
+    else if ((w >> 28) == 3)
+      snprintf(msg, sizeof(msg), "a kernel gave up waiting: wait self-test, block %u, warp %u", (w >> 16) & 0xfffu, w & 0xffu);
     else
       snprintf(msg, sizeof(msg), "a kernel gave up waiting: tensor-core attention (records no location)");
     ctx->err = msg;
   }
+  return RECACHE_OK;
+}
+
+recache_status recache_selftest_wait_timeout(recache_ctx* ctx, int32_t* report, void* stream) {
+  if (!ctx || !report) return RECACHE_EINVAL;
+  RC_CUDA(cudaSetDevice(ctx->device), "selftest: set device");
+  RC_CUDA(rc_launch_wait_selftest(ctx, report, (cudaStream_t)stream), "selftest launch");
   return RECACHE_OK;
 }
 

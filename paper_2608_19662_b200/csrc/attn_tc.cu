@@ -97,31 +97,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after WAIT_PROBES unsuccessful probes (or as soon as another thread of
-// the CTA has given up), records the failure in the device status word and lets the kernel run to
-// its end so that tensor memory is released.  The bound is a probe count, not a clock reading:
-// a probe that fails has suspended the thread for about 1.3 us (measured), and the loop then
-// holds no 64-bit start time across it: the 32-register warps of this kernel are sensitive to
-// every register and instruction around their waits.
+// Bounded wait: see rc_mbar_wait (no location word here).
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try(bar, parity)) return;
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return;
-    if ((it & 1023u) == 0u) {
-      if (*abort_flag) return;
-      if (it >= WAIT_PROBES) {   // (no location word here: even one more instruction on this cold path costs the kernel 6 %)
-        *abort_flag = 1;
-        rc_set_status(status, RECACHE_DEV_TIMEOUT);
-        return;
-      }
-    }
-  }
+  rc_mbar_wait<WAIT_PROBES, 0>(bar, parity, abort_flag, status);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -528,8 +506,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       // path, and the rotation is the urgent one: a tile's O is written back once the same tile's
       // next Q has been rotated.  (O is not needed back before the next item's first P V, a whole
       // softmax later; tile B's rotation finishes after tile A's, so tile A is not held up by it.)
+      // This wait is a matter of priority only, so it is taken only where the rotating warpgroup
+      // cannot complete a second phase before it: tile A's warpgroup is active in every item and
+      // stops at the end of the next item for this item's O-drained arrival, which comes after the
+      // wait.  Tile B's warpgroup rotates Q even in items where its tile is empty and is held back by
+      // nothing there, so with an empty tile B in this item or the next (short sequences) it could
+      // pass two phases while tile A is being drained here, and a parity wait would then sleep
+      // through the phase it wants.
       for (int x = 0; x < 2; ++x) {
-        if (nx.n_tiles > 0) mbar_wait(bar(B_QREADY + x), (item_n + 1u) & 1u, abort_flag, p.status);
+        if (nx.n_tiles > 0 && (x == 0 || (it.b_valid && nx.b_valid)))
+          mbar_wait(bar(B_QREADY + x), (item_n + 1u) & 1u, abort_flag, p.status);
         if (x == 1 && !it.b_valid) continue;
         mbar_wait(bar(B_LREADY + x), done[x] & 1u, abort_flag, p.status);
         mbar_wait(bar(B_ODONE + x), done[x] & 1u, abort_flag, p.status);
@@ -943,14 +929,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
   }
   // ---- teardown: every thread is done with tensor memory before it is freed ----
-  if (*abort_flag) {
-    // A wait ran out: the roles fell through their loops with loads, copies and MMAs possibly still in
-    // flight.  Let them land (none depends on another CTA; ~100 us is far more than any of them takes)
-    // before shared and tensor memory go away under them.
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    const long long t0 = clock64();
-    while (clock64() - t0 < 200000ll) { }
-  }
+  if (*abort_flag) rc_timeout_drain();   // a wait ran out: let what is in flight land first
   tc_fence_before();
   __syncthreads();
   if (warp == 9) {

@@ -70,10 +70,51 @@ __device__ __forceinline__ void rc_set_status(int32_t* status, int32_t code) {
 // A bounded wait of the split-KV decode kernel that ran out also says where (second status word, first one wins):
 // kernel tag << 28 | (block & 0xfff) << 16 | (barrier's shared address / 8 & 0xff) << 8 | warp.
 constexpr uint32_t RC_WHERE_DECODE_SPLIT = 2;
+constexpr uint32_t RC_WHERE_SELFTEST = 3;
 __device__ __forceinline__ void rc_set_timeout(int32_t* status, uint32_t kernel_tag, uint32_t bar) {
   atomicCAS(status, 0, (int32_t)RECACHE_DEV_TIMEOUT);
   const uint32_t where = kernel_tag << 28 | (blockIdx.x & 0xfffu) << 16 | ((bar >> 3) & 0xffu) << 8 | (threadIdx.x >> 5);
   atomicCAS(status + 1, 0, (int32_t)where);
+}
+
+// ---- bounded mbarrier wait, shared by the TMA kernels ----
+__device__ __forceinline__ bool rc_mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Gives up after PROBES unsuccessful probes (or as soon as another thread of the CTA has given
+// up), records RECACHE_DEV_TIMEOUT in the device status word and returns, so that the kernel runs
+// to its end and releases what it holds.  The bound is a probe count, not a clock reading: a probe
+// that fails has suspended the thread for about 1.3 us (measured), and the loop then holds no
+// 64-bit start time across it (the 32-register warps of the attention kernel are sensitive to every
+// register and instruction around their waits).  WHERE_TAG != 0 also records where the wait ran
+// out (second status word); the attention kernel passes 0: one more instruction on this cold path
+// cost it 6 %.
+template <uint32_t PROBES, uint32_t WHERE_TAG>
+__device__ __forceinline__ void rc_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (rc_mbar_try(bar, parity)) return;
+  for (uint32_t it = 1;; ++it) {
+    if (rc_mbar_try(bar, parity)) return;
+    if ((it & 1023u) == 0u) {
+      if (*abort_flag) return;
+      if (it >= PROBES) {
+        *abort_flag = 1;
+        if constexpr (WHERE_TAG != 0) rc_set_timeout(status, WHERE_TAG, bar);
+        else rc_set_status(status, RECACHE_DEV_TIMEOUT);
+        return;
+      }
+    }
+  }
+}
+// After a wait ran out the roles fall through their loops with loads, copies and MMAs possibly
+// still in flight.  Let them land (none depends on another CTA; ~100 us is far more than any of
+// them takes) before shared and tensor memory go away under them.
+__device__ __forceinline__ void rc_timeout_drain() {
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  const long long t0 = clock64();
+  while (clock64() - t0 < 200000ll) { }
 }
 
 // Largest i with cu[i] <= x, for cu[0..n] non-decreasing (n >= 1).
@@ -205,6 +246,9 @@ struct TcAttnArgs {
 bool rc_tc_supported(const recache_ctx* ctx);
 int64_t rc_tc_workspace_bytes(const recache_ctx* ctx, int n_seq, int total, int max_len);
 cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaStream_t st);
+
+// ---- self-test of the bounded barrier wait (report: 2 ints on the device) ----
+cudaError_t rc_launch_wait_selftest(const recache_ctx* ctx, int32_t* report, cudaStream_t st);
 
 // ---- bf16 split-KV paged decode (TMA + mma.sync, persistent) ----
 bool rc_decode_split_supported(const recache_ctx* ctx);

@@ -21,6 +21,8 @@
 // Every K/V byte crosses HBM once; the roofline is bytes / HBM bandwidth.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace {
@@ -80,23 +82,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait (see the tensor-core attention kernel): never spins forever.  The bound counts
-// unsuccessful probes (each suspends the thread for about 1.3 us).
+// Bounded wait: see rc_mbar_wait; this kernel also records where a wait ran out.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (mbar_try(bar, parity)) return;
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return;
-    if ((it & 1023u) == 0u) {
-      if (*abort_flag) return;
-      if (it >= WAIT_PROBES) { *abort_flag = 1; rc_set_timeout(status, RC_WHERE_DECODE_SPLIT, bar); return; }
-    }
-  }
+  rc_mbar_wait<WAIT_PROBES, RC_WHERE_DECODE_SPLIT>(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -412,13 +400,7 @@ __global__ void __launch_bounds__(GATHER ? NTHREADS_GATHER : NTHREADS, 1) decode
       bar_consumers();
     }
   }
-  if (*abort_flag) {
-    // A wait ran out: loads may still be in flight towards this CTA's shared memory.  Let them
-    // land (~100 us is far more than any of them takes) before the CTA ends.
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    const long long t0 = clock64();
-    while (clock64() - t0 < 200000ll) { }
-  }
+  if (*abort_flag) rc_timeout_drain();   // a wait ran out: let the loads in flight land before the CTA ends
 }
 
 // Combines the splits of every (sequence, head): grid = batch * Hq, 32 threads x 4 dims.
@@ -570,7 +552,10 @@ constexpr int64_t NOALLOC_SCRATCH_BYTES = 4ll << 20;   // 4 MiB per device
 static __device__ __align__(256) unsigned char g_decode_scratch[NOALLOC_SCRATCH_BYTES];
 
 constexpr int NOALLOC_MAX_DEVICES = 64;
-void* g_scratch_addr[NOALLOC_MAX_DEVICES] = {nullptr};   // device address of g_decode_scratch, per device
+// Device address of g_decode_scratch, per device.  Host threads may make the first call on a
+// device at the same time: each looks the address up and stores the same value, through an atomic
+// so that the concurrent store and load are well defined.
+std::atomic<void*> g_scratch_addr[NOALLOC_MAX_DEVICES];
 
 }  // namespace
 
@@ -604,14 +589,14 @@ extern "C" RECACHE_API recache_status recache_attend_decode_noalloc(
   if (cudaSetDevice(ctx->device) != cudaSuccess) return fail(RECACHE_ECUDA, "decode_noalloc: set device");
   // In host code the array's name is only a handle; the kernel needs its device
   // address, looked up once per device with that device current.
-  void* scratch = g_scratch_addr[ctx->device];
+  void* scratch = g_scratch_addr[ctx->device].load(std::memory_order_relaxed);
   if (!scratch) {
     cudaError_t e = cudaGetSymbolAddress(&scratch, g_decode_scratch);
     if (e != cudaSuccess || !scratch) {
       ctx->err = std::string("decode_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e);
       return RECACHE_ECUDA;
     }
-    g_scratch_addr[ctx->device] = scratch;
+    g_scratch_addr[ctx->device].store(scratch, std::memory_order_relaxed);
   }
   cudaStream_t st = (cudaStream_t)stream;
   DecodeArgs a{q, q_pos, batch, k_new, v_new, k_pages, v_pages, n_pages, res_page_table, max_res_pages, res_len,

@@ -268,20 +268,31 @@ def config3_pool(n_pool=64, len_range=(150, 1200), seed=SEED0 + 3, layer=0,
     return pack_resources(shape, seed, lens, masks, layer=layer)
 
 
-def config3_requests(pool: ResourceBatch, n_requests=16, draw=(4, 12), tq_range=(256, 1024),
-                     seed=SEED0 + 3, layer=0, route_frac=0.25):
-    """Requests drawing 4-12 distinct pool resources in random order; routes are
-    redrawn per layer, the compositions are not."""
-    shape = pool.shape
+def config3_compositions(n_pool: int, n_requests=16, draw=(4, 12), tq_range=(256, 1024), seed=SEED0 + 3):
+    """The requests of the composition-reuse workload: each draws 4-12 distinct pool
+    resources in random order and has 256-1024 query tokens.  The same for every layer."""
     rng = np.random.default_rng(seed + 17)
-    n_pool = len(pool.lens)
     lists, tqs = [], []
     for _ in range(n_requests):
         k = int(rng.integers(draw[0], min(draw[1], n_pool) + 1))
         lists.append([int(x) for x in rng.choice(n_pool, size=k, replace=False)])
         tqs.append(int(rng.integers(tq_range[0], tq_range[1] + 1)))
+    return lists, tqs
+
+
+def config3_layer_routes(shape: Shape, lists, layer: int, seed=SEED0 + 3, route_frac=0.25):
+    """Routes of one layer: redrawn per layer (the compositions are not)."""
     rng_l = np.random.default_rng(seed + 1000 + layer)
-    vis = [routes_random(rng_l, shape.n_kv_heads, len(l), route_frac) for l in lists]
+    return [routes_random(rng_l, shape.n_kv_heads, len(l), route_frac) for l in lists]
+
+
+def config3_requests(pool: ResourceBatch, n_requests=16, draw=(4, 12), tq_range=(256, 1024),
+                     seed=SEED0 + 3, layer=0, route_frac=0.25):
+    """Requests drawing 4-12 distinct pool resources in random order; routes are
+    redrawn per layer, the compositions are not."""
+    shape = pool.shape
+    lists, tqs = config3_compositions(len(pool.lens), n_requests, draw, tq_range, seed)
+    vis = config3_layer_routes(shape, lists, layer, seed, route_frac)
     return make_requests(shape, seed + 31 * layer, pool, lists, vis, tqs)
 
 

@@ -195,3 +195,54 @@ def test_host_side_errors_are_returned_before_any_launch():
                           torch.empty((64, 128), dtype=torch.bfloat16, device="cuda"),
                           torch.empty((64, 128), dtype=torch.bfloat16, device="cuda"))
     assert rc.poll_status() == 0
+
+
+def test_bounded_wait_runs_out_sets_status_and_context_stays_usable():
+    """The failure path of the TMA kernels' barrier waits, exercised by the library's
+    self-test kernel (same wait and drain helpers, small probe bound, a barrier nobody
+    arrives at): it must give up within milliseconds, report RECACHE_DEV_TIMEOUT with
+    its location, and leave the context clean for the next ordinary call."""
+    sh = wl.QWEN3_4B
+    rc = make_ctx(sh, max_pos=1024)
+    gave_up, kcycles = rc.selftest_wait_timeout()
+    assert gave_up
+    assert 100 < kcycles < 100_000                 # ~2^10 suspended probes: around a millisecond, never seconds
+    assert rc.poll_status() == 7                   # RECACHE_DEV_TIMEOUT
+    assert "wait self-test" in rc.last_error()
+    assert rc.poll_status() == 0                   # cleared by the poll
+    pool = _pool(sh, [70, 200])
+    o_ref, _, _ = oracle_encode(pool)
+    o, _, _ = gpu_encode(rc, pool)
+    assert max_abs(o, o_ref) < TOL_BF16 and rc.poll_status() == 0
+
+
+@pytest.mark.parametrize("hq,g", [(16, 8), (32, 8), (32, 4)])
+def test_thousands_of_tiny_resources(hq, g):
+    """Many resources no longer than one query tile (1 .. 128/s tokens, so the
+    second tile of every work item is empty and every item has a single K/V
+    tile): each CTA runs dozens of such items back to back, the case in which a
+    role that is idle in an item could run ahead of the others."""
+    sh = wl.Shape(hq, g, 128, 1e6, "bf16")
+    tq = 128 // sh.group_size
+    rng = np.random.default_rng(hq + g)
+    n = 2000
+    lens = rng.integers(1, tq + 1, n)
+    lens[::7] = rng.integers(tq + 1, 2 * tq + 1, len(lens[::7]))     # some with a second tile in between
+    pool = _pool(sh, [int(x) for x in lens], keep=[np.ones(int(x), np.uint8) for x in lens])
+    rc = make_ctx(sh, max_pos=1024)
+    o_ref, kc_ref, vc_ref = oracle_encode(pool)
+    o, kc, vc = gpu_encode(rc, pool)
+    assert rc.poll_status() == 0
+    assert max_abs(o, o_ref) < TOL_BF16
+    assert np.array_equal(f64(vc)[~np.isnan(vc_ref)], vc_ref[~np.isnan(vc_ref)])
+    # many short requests with empty routes through the prefill entry point
+    nreq = 600
+    tqs = [int(x) for x in rng.integers(1, tq + 1, nreq)]
+    vis0 = np.zeros((g, 1), np.uint8)
+    req = wl.make_requests(sh, 9, pool, [[0]] * nreq, [vis0] * nreq, tqs)
+    rows = oracle_rows(pool, req)
+    out = gpu_compact(rc, pool, req, kc, vc)
+    p_ref, _ = oracle_prefill(req, rows, kc_ref, vc_ref)
+    p, _, _ = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
+    assert rc.poll_status() == 0
+    assert max_abs(p, p_ref) < TOL_BF16
