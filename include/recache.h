@@ -7,7 +7,7 @@
  * conversation sees, on every (layer, KV-head-group) route, only the resources
  * that route exposes ("Structural Pruning", masks M_resource / M_context) and
  * only their retained token fields ("Semantic Pruning"); the gather of those
- * rows is the "request-local KV materialization" the paper counts inside TTFT
+ * rows is the request-local materialisation of KV that the paper counts inside TTFT
  * (section "Evaluation Metrics", paragraph "Efficiency").
  *
  * Conventions that hold for every call
@@ -170,13 +170,13 @@ RECACHE_API recache_status recache_encode_resources(recache_ctx* ctx,
 
 /*
  * Encoding variants of the paper's ablation (section "Cache Reuse"): resources
- * "pre-encoded with a shared prefix", and the "Block" configuration that drops
- * cross-resource attention but keeps the original positional indices.
+ * encoded behind a prefix they all share, and the Block configuration, which
+ * has no attention between resources but leaves every token at its global position.
  * Same as recache_encode_resources, plus
  *   k_prefix / v_prefix [G][prefix_len][d]: rotated keys and values of a shared
  *       prefix, as a cache holds them (e.g. written by an earlier encode call);
- *       every resource token also attends to all of them ("attend only to the
- *       shared prefix and their local resource tokens").  NULL / 0: no prefix.
+ *       every resource token also attends to all of them (the shared-prefix form
+ *       of section "Resource-Wise Attention").  NULL / 0: no prefix.
  *   pos_offset [N] (device, may be NULL = all 0): position of each resource's
  *       first token.  One common value P = the resource-local layout behind a
  *       prefix of P tokens (still composition-independent); global offsets = the
@@ -251,8 +251,8 @@ RECACHE_API recache_status recache_attend_prefill(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
- * Routed prefill of a later turn (paper, problem setup: the input also holds the
- * "preceding conversational history when available in multi-turn interactions").
+ * Routed prefill of a later turn (paper, problem setup: in a multi-turn
+ * interaction the input also carries the turns that came before).
  * Same as recache_attend_prefill, with the conversation's rotated keys / values
  * kept in a cache [G][cache_rows][d]: request b owns rows conv_slot[b] ..., of
  * which the first hist_len[b] hold its earlier turns.  The new tokens attend to
@@ -295,7 +295,7 @@ RECACHE_API recache_status recache_attend_prefill_gather(recache_ctx* ctx,
     void* workspace, int64_t workspace_bytes, void* stream);
 
 /*
- * Routed decode (paper: the same mask "during decoding"; the Attn. latency of
+ * Routed decode (paper: the final mask also holds while decoding; the Attn. latency of
  * the efficiency study).  One query token per sequence at position q_pos[b].
  * Item it = b * G + g reads res_len[it] rows through res_page_table[it][*] and
  * hist_len[it] rows through hist_page_table[it][*] (row n lives in page
@@ -322,6 +322,9 @@ RECACHE_API recache_status recache_attend_decode(recache_ctx* ctx,
  * to get the indices only: no key / value byte is moved, and requests that share
  * a resource share its cache rows).  History stays paged as in
  * recache_attend_decode; same softmax, same results.
+ *   route_rows: number of entries of route_idx (an item whose route_cu range does
+ *   not lie inside it is reported as RECACHE_DEV_OVERFLOW and read as an empty route);
+ *   pool_tokens > 0;
  *   max_res_pages: upper bound of ceil(route length / page_tokens), used to size
  *   the split plan and the workspace (recache_decode_workspace_bytes).
  * bf16 contexts with head_dim 128 and 64-token pages only.
@@ -330,7 +333,7 @@ RECACHE_API recache_status recache_attend_decode_gather(recache_ctx* ctx,
     const void* q, const int32_t* q_pos, int32_t batch,
     const void* k_new, const void* v_new,
     const void* k_cache, const void* v_cache, int64_t pool_tokens,
-    const int32_t* route_idx, const int32_t* route_cu, int32_t max_res_pages,
+    const int32_t* route_idx, const int32_t* route_cu, int64_t route_rows, int32_t max_res_pages,
     void* k_pages, void* v_pages, int64_t n_pages,
     const int32_t* hist_page_table, int32_t max_hist_pages, const int32_t* hist_len,
     void* out_o, int32_t out_dtype,

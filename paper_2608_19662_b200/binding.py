@@ -58,7 +58,7 @@ SIGNATURES = {
                                                  _I64, _P, _P, _P, _I32, _P, _I64, _P]),
     "recache_attend_decode": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _I32, _P, _P, _I32, _P,
                                         _P, _I32, _P, _I64, _P]),
-    "recache_attend_decode_gather": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _P, _I32, _P, _P, _I64,
+    "recache_attend_decode_gather": (C.c_int, [_P, _P, _P, _I32, _P, _P, _P, _P, _I64, _P, _P, _I64, _I32, _P, _P, _I64,
                                                _P, _I32, _P, _P, _I32, _P, _I64, _P]),
     "recache_build_routes": (C.c_int, [C.POINTER(C.c_double), _I32, C.POINTER(C.c_double), _I32, _I32, _I32,
                                        C.POINTER(C.c_uint8), C.POINTER(C.c_double), C.POINTER(C.c_double),
@@ -345,7 +345,8 @@ class ReCache:
         ws = workspace if workspace is not None else self.workspace(self.decode_workspace_bytes(batch, max_res_pages, mh))
         st = self.lib.recache_attend_decode_gather(
             self.h, _ptr(q), _ptr(q_pos), batch, _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), k_cache.shape[1],
-            _ptr(route_idx), _ptr(route_cu), int(max_res_pages), _ptr(k_pages), _ptr(v_pages), k_pages.shape[0],
+            _ptr(route_idx), _ptr(route_cu), route_idx.numel(), int(max_res_pages), _ptr(k_pages), _ptr(v_pages),
+            k_pages.shape[0],
             _ptr(hist_page_table), mh, _ptr(hist_len), _ptr(out), oc, _ptr(ws), ws.numel(), _stream())
         self._check(st, "recache_attend_decode_gather")
         return out

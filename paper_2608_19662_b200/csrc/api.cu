@@ -373,14 +373,15 @@ recache_status recache_attend_decode(recache_ctx* ctx, const void* q, const int3
 recache_status recache_attend_decode_gather(recache_ctx* ctx, const void* q, const int32_t* q_pos, int32_t batch,
                                             const void* k_new, const void* v_new, const void* k_cache,
                                             const void* v_cache, int64_t pool_tokens, const int32_t* route_idx,
-                                            const int32_t* route_cu, int32_t max_res_pages, void* k_pages,
+                                            const int32_t* route_cu, int64_t route_rows, int32_t max_res_pages, void* k_pages,
                                             void* v_pages, int64_t n_pages, const int32_t* hist_page_table,
                                             int32_t max_hist_pages, const int32_t* hist_len, void* out_o,
                                             int32_t out_dtype, void* workspace, int64_t workspace_bytes,
                                             void* stream) {
   if (!ctx) return RECACHE_EINVAL;
-  RC_REQUIRE(batch >= 0 && n_pages >= 0 && max_res_pages >= 0 && max_hist_pages > 0 && pool_tokens >= 0,
+  RC_REQUIRE(batch >= 0 && n_pages >= 0 && max_res_pages >= 0 && max_hist_pages > 0 && pool_tokens >= 0 && route_rows >= 0,
              RECACHE_EINVAL, "decode_gather: bad size");
+  RC_REQUIRE(batch == 0 || pool_tokens > 0, RECACHE_EINVAL, "decode_gather: an index list needs a cache with at least one row");
   RC_REQUIRE(out_dtype_ok(ctx, out_dtype), RECACHE_EINVAL, "decode_gather: out_dtype must be f32 or the context dtype");
   RC_REQUIRE(rc_decode_split_supported(ctx), RECACHE_EUNSUPPORTED,
              "decode_gather: needs a bf16 context with head_dim 128 and 64-token pages");
@@ -397,6 +398,7 @@ recache_status recache_attend_decode_gather(recache_ctx* ctx, const void* q, con
   DecodeArgs a{q, q_pos, batch, k_new, v_new, k_pages, v_pages, n_pages, nullptr, max_res_pages, nullptr,
                hist_page_table, max_hist_pages, hist_len, out_o, out_dtype, workspace, workspace_bytes};
   a.k_cache = k_cache; a.v_cache = v_cache; a.pool_tokens = pool_tokens; a.route_idx = route_idx; a.route_cu = route_cu;
+  a.route_rows = route_rows;
   if (k_new) RC_CUDA(rc_launch_decode_append(ctx, a, st), "decode_gather: append launch");
   RC_CUDA(rc_launch_decode_split(ctx, a, st), "decode_gather: attention launch");
   return RECACHE_OK;

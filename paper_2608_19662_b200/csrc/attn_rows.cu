@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
     const int32_t* __restrict__ pos0, const int32_t* __restrict__ slot,
     const T* __restrict__ k_self, const T* __restrict__ v_self, int64_t self_rows,
     const T* __restrict__ k_route, const T* __restrict__ v_route, const int32_t* __restrict__ route_cu,
-    int prefix_len, const int32_t* __restrict__ hist, int Hq, int G, const float* __restrict__ cos_tab, const float* __restrict__ sin_tab, int max_pos,
+    int prefix_len, const int32_t* __restrict__ hist, int64_t route_rows, int Hq, int G, const float* __restrict__ cos_tab, const float* __restrict__ sin_tab, int max_pos,
     float scale, int32_t* status) {
   __shared__ float q_s[WARPS][D];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -94,6 +94,12 @@ __global__ void __launch_bounds__(WARPS * 32) attn_rows_kernel(
       // the route's packed rows, or (encoding behind a shared prefix) the group's prefix rows
       const int r0 = route_cu ? route_cu[b * G + g] : g * prefix_len;
       const int r1 = route_cu ? route_cu[b * G + g + 1] : r0 + prefix_len;
+      // a range outside the route tensors (e.g. after a compaction that overflowed its capacity)
+      // is reported and read as an empty route
+      if (r0 < 0 || r1 < r0 || (int64_t)r1 > route_rows) {
+        if (lane == 0) rc_set_status(status, RECACHE_DEV_OVERFLOW);
+        continue;
+      }
       kb = k_route + (int64_t)r0 * D; vb = v_route + (int64_t)r0 * D; n = r1 - r0;
     } else {
       kb = k_self + ((int64_t)g * self_rows + base) * D;
@@ -141,7 +147,7 @@ cudaError_t launch(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t s
   const float scale = (float)(1.0 / sqrt((double)d));
   RcLaunchScope scope(ctx, a.route_cu ? RC_K_PREFILL_ATTN : RC_K_ENCODE_ATTN, st);
 #define RC_ARGS (const T*)a.q, (TO*)a.o, a.cu, a.n_seq, a.total, a.pos0, a.slot, (const T*)a.k_self, \
-    (const T*)a.v_self, a.self_rows, (const T*)a.k_route, (const T*)a.v_route, a.route_cu, a.prefix_len, a.hist, Hq, G, \
+    (const T*)a.v_self, a.self_rows, (const T*)a.k_route, (const T*)a.v_route, a.route_cu, a.prefix_len, a.hist, a.route_rows, Hq, G, \
     ctx->cos_tab, ctx->sin_tab, ctx->desc.max_pos, scale, ctx->status
   if (d == 64) attn_rows_kernel<T, TO, 64><<<blocks, WARPS * 32, 0, st>>>(RC_ARGS);
   else         attn_rows_kernel<T, TO, 128><<<blocks, WARPS * 32, 0, st>>>(RC_ARGS);

@@ -79,6 +79,7 @@ struct TcParams {
   int n_seq, G, Hq, s;
   int prefix_len;   // > 0: every sequence sees rows g*prefix_len .. of the "route" tensors (shared prefix)
   int64_t self_rows;
+  int64_t route_rows;   // rows of the packed route tensors / entries of route_idx
   void* out;
   const float* cos_tab; const float* sin_tab; int max_pos;
   float scale_log2;
@@ -263,13 +264,17 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
   it.base = p.slot ? (int64_t)p.slot[b] : (int64_t)it.seq0;
   it.pos0 = p.pos0 ? p.pos0[b] : 0;
   it.rA0 = 0; it.lenA = 0;
-  if (p.route_cu) { it.rA0 = p.route_cu[b * p.G + it.g]; it.lenA = p.route_cu[b * p.G + it.g + 1] - it.rA0; }
+  bool route_ok = true;
+  if (p.route_cu) {
+    it.rA0 = p.route_cu[b * p.G + it.g]; it.lenA = p.route_cu[b * p.G + it.g + 1] - it.rA0;
+    route_ok = (int64_t)it.rA0 + it.lenA <= p.route_rows;   // e.g. after a compaction that overflowed its capacity
+  }
   else if (p.prefix_len > 0) { it.rA0 = it.g * p.prefix_len; it.lenA = p.prefix_len; }
   it.nA = (it.lenA + TILE_N - 1) / TILE_N;
   it.n_tiles = it.nA + (it.kv_end + TILE_N - 1) / TILE_N;
   const bool ok = it.L > 0 && it.tok0 < it.L && it.lenA >= 0 && it.rA0 >= 0 && it.base >= 0 && it.H >= 0 &&
-                  it.base + it.H + it.L <= p.self_rows && it.seq0 >= 0;
-  if (!ok) rc_set_status(p.status, RECACHE_DEV_BAD_SLOT);
+                  it.base + it.H + it.L <= p.self_rows && it.seq0 >= 0 && route_ok;
+  if (!ok) rc_set_status(p.status, route_ok ? RECACHE_DEV_BAD_SLOT : RECACHE_DEV_OVERFLOW);
   return ok;
 }
 
@@ -1028,7 +1033,7 @@ cudaError_t rc_launch_attn_tc(const recache_ctx* ctx, const TcAttnArgs& a, cudaS
 
   TcParams p;
   p.items = items; p.header = header; p.cu = a.cu; p.pos0 = a.pos0; p.slot = a.slot; p.route_cu = a.route_cu;
-  p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.out = a.o;
+  p.n_seq = a.n_seq; p.G = G; p.Hq = Hq; p.s = s; p.self_rows = a.self_rows; p.route_rows = a.route_rows; p.out = a.o;
   p.prefix_len = a.route_cu ? 0 : a.prefix_len;
   p.hist = a.hist;
   p.cos_tab = ctx->cos_tab; p.sin_tab = ctx->sin_tab; p.max_pos = ctx->desc.max_pos;

@@ -166,6 +166,7 @@ struct AttnRowsArgs {
   const void* k_route; const void* v_route; const int32_t* route_cu;  // null for encode
   int prefix_len;   // > 0 (with route_cu null): every sequence sees rows g*prefix_len .. +prefix_len of k_route/v_route
   const int32_t* hist = nullptr;   // rows that precede each sequence's own tokens in the self part, all visible
+  int64_t route_rows = 0;          // rows of k_route / v_route: a route_cu range outside them is reported and skipped
 };
 cudaError_t rc_launch_attn_rows(const recache_ctx* ctx, const AttnRowsArgs& a, cudaStream_t st);
 
@@ -196,6 +197,7 @@ struct DecodeArgs {
   // route_idx[route_cu[it] .. route_cu[it+1]) of the cache; res_pt / res_len are unused
   const void* k_cache = nullptr; const void* v_cache = nullptr; int64_t pool_tokens = 0;
   const int32_t* route_idx = nullptr; const int32_t* route_cu = nullptr;
+  int64_t route_rows = 0;   // entries of route_idx
 };
 cudaError_t rc_launch_decode_append(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);
 cudaError_t rc_launch_decode_rows(const recache_ctx* ctx, const DecodeArgs& a, cudaStream_t st);

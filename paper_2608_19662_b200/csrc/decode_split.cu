@@ -69,7 +69,7 @@ struct DecParams {
   int32_t* status;
   // gather variant: the resource part of item `it` is rows route_idx[route_cu[it] .. route_cu[it+1]) of the cache
   const __nv_bfloat16* k_cache; const __nv_bfloat16* v_cache; int64_t pool_tokens;
-  const int32_t* route_idx; const int32_t* route_cu;
+  const int32_t* route_idx; const int32_t* route_cu; int64_t route_rows;   // entries of route_idx
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -125,7 +125,15 @@ struct UnitPages { int n_res_pages, n_hist_pages, p0, p1, res_len, hist_len; };
 template <bool GATHER>
 __device__ __forceinline__ UnitPages unit_pages(const DecParams& p, int it, int sp) {
   UnitPages u;
-  u.res_len = GATHER ? max(p.route_cu[it + 1] - p.route_cu[it], 0) : max(p.res_len[it], 0);
+  if (GATHER) {
+    // the item's slice of the index list must lie inside it; otherwise the route is treated as empty
+    const int r0 = p.route_cu[it], r1 = p.route_cu[it + 1];
+    const bool ok = r0 >= 0 && r1 >= r0 && (int64_t)r1 <= p.route_rows;
+    if (!ok) rc_set_status(p.status, RECACHE_DEV_OVERFLOW);
+    u.res_len = ok ? r1 - r0 : 0;
+  } else {
+    u.res_len = max(p.res_len[it], 0);
+  }
   u.hist_len = max(p.hist_len[it], 0);
   u.n_res_pages = GATHER ? (u.res_len + PT - 1) / PT : min((u.res_len + PT - 1) / PT, p.max_res_pages);
   u.n_hist_pages = min((u.hist_len + PT - 1) / PT, p.max_hist_pages);
@@ -509,7 +517,7 @@ cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, 
   p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)D));
   p.status = ctx->status;
   p.k_cache = (const __nv_bfloat16*)a.k_cache; p.v_cache = (const __nv_bfloat16*)a.v_cache;
-  p.pool_tokens = a.pool_tokens; p.route_idx = a.route_idx; p.route_cu = a.route_cu;
+  p.pool_tokens = a.pool_tokens; p.route_idx = a.route_idx; p.route_cu = a.route_cu; p.route_rows = a.route_rows;
   const int sms = ctx->sm_count > 0 ? ctx->sm_count : 148;
   const unsigned grid = (unsigned)(units < sms ? units : sms);
   const bool f32 = a.out_dtype == RECACHE_F32, gather = a.route_idx != nullptr;

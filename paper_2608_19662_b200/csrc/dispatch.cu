@@ -24,6 +24,7 @@ cudaError_t rc_launch_encode_attn(const recache_ctx* ctx, const EncodeArgs& a, c
   }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu, a.n_res, a.total, a.pos_offset, a.slot, a.k_cache, a.v_cache,
                  a.pool_tokens, a.k_prefix, a.v_prefix, nullptr, a.prefix_len};
+  r.route_rows = (int64_t)ctx->desc.n_kv_heads * a.prefix_len;
   return rc_launch_attn_rows(ctx, r, st);
 }
 
@@ -36,6 +37,7 @@ cudaError_t rc_launch_prefill_attn(const recache_ctx* ctx, const PrefillArgs& a,
   }
   AttnRowsArgs r{a.q, a.o, a.out_dtype, a.cu_q, a.n_req, a.total_q, a.pos0, a.conv_slot, a.k_conv, a.v_conv,
                  a.conv_rows, a.k_route, a.v_route, a.route_cu, 0, a.hist};
+  r.route_rows = a.route_rows;
   return rc_launch_attn_rows(ctx, r, st);
 }
 

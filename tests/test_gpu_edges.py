@@ -153,6 +153,20 @@ def test_device_status_codes_instead_of_faults():
     out = gpu_compact(rc, wl.keep_all(pool), req, kc, vc, capacity=100)
     assert rc.poll_status() == 3
     assert int(out["route_cu"][-1]) == 110 * sh.n_kv_heads
+    # a prefill handed that prefix (ranges beyond the 100 packed rows) reports it and skips those routes,
+    # on the tensor-core path and on the exact row-per-warp path alike
+    gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"])
+    assert rc.poll_status() == 3
+    sh32 = wl.Shape(4, 2, 64, 1e4, "f32")
+    pool32 = wl.keep_all(_pool(sh32, [50, 60]))
+    rc32 = make_ctx(sh32, max_pos=1024)
+    _, kc32, vc32 = gpu_encode(rc32, pool32)
+    vis32 = np.ones((sh32.n_kv_heads, 2), np.uint8)
+    req32 = wl.make_requests(sh32, 3, pool32, [[0, 1]], [vis32], [8])
+    out32 = gpu_compact(rc32, pool32, req32, kc32, vc32, capacity=100)
+    assert rc32.poll_status() == 3
+    gpu_prefill(rc32, req32, out32["k_out"], out32["v_out"], out32["route_cu"])
+    assert rc32.poll_status() == 3
     # conversation positions running past the rotary table (1000 + 64 > 1024)
     req_far = wl.make_requests(sh, 4, wl.keep_all(pool), [[0, 1]], [vis], [64], q_pos0=[1000])
     big = gpu_compact(rc, wl.keep_all(pool), req_far, kc, vc)

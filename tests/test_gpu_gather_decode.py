@@ -78,3 +78,9 @@ def test_gather_decode_equals_paged_decode_and_oracle(batch, n_res, res_len, his
                                 hist_t, hl, sh.rope_theta, pt, storage="bf16")
         assert np.abs(f64(o_g[b, kg * s:(kg + 1) * s]) - ref[0]).max() < 1e-2
     assert rc.poll_status() == 0
+    # an index list shorter than the prefix says: the items past its end are reported and read as empty
+    # routes (history only), nothing is read outside the list
+    short = r_idx[:int(cu[n_items // 2])].clone()
+    rc.attend_decode_gather(dev(q), dev(dc.q_pos), kc, vc, short, r_cu, dc.max_res_pages, kp1, vp1,
+                            dev(dc.hist_page_table), dev(dc.hist_len), out_dtype=torch.float32)
+    assert rc.poll_status() == 3
