@@ -86,6 +86,19 @@ struct TcParams {
   int32_t* status;
 };
 
+// Optional in-kernel timeline (build with -DRC_TRACE; never part of the shipped library): CTA 0
+// stamps %clock64 at the hand-overs of its first TR_ITEMS work items, one row of 16 stamps per
+// (role, item).  Without the flag the macro is empty.
+#ifdef RC_TRACE
+constexpr int TR_ITEMS = 192, TR_ROLES = 5;   // roles: softmax A, softmax B, MMA, epilogue, producer
+__device__ long long g_trace[TR_ROLES * TR_ITEMS * 16];
+#define TR(role, item, k) do { if (blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = clock64(); } while (0)
+#define TRV(role, item, k, v) do { if (blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = (v); } while (0)
+#else
+#define TR(role, item, k) do {} while (0)
+#define TRV(role, item, k, v) do {} while (0)
+#endif
+
 // ------------------------------------------------------------------ PTX --
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -507,6 +520,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         kv_n += (uint32_t)it.n_tiles;
       }
       fetch_item(item_n + 1, nx, true);
+      if (row == 0) { TR(3, item_n, 0); TRV(3, item_n, 15, it.n_tiles * 2 + it.b_valid); }
       // The stores below and the rotation of the next item's Q go through the same load/store
       // path, and the rotation is the urgent one: a tile's O is written back once the same tile's
       // next Q has been rotated.  (O is not needed back before the next item's first P V, a whole
@@ -521,9 +535,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       for (int x = 0; x < 2; ++x) {
         if (nx.n_tiles > 0 && (x == 0 || (it.b_valid && nx.b_valid)))
           mbar_wait(bar(B_QREADY + x), (item_n + 1u) & 1u, abort_flag, p.status);
+        if (row == 0) TR(3, item_n, 1 + 5 * x);
         if (x == 1 && !it.b_valid) continue;
         mbar_wait(bar(B_LREADY + x), done[x] & 1u, abort_flag, p.status);
+        if (row == 0) TR(3, item_n, 2 + 5 * x);
         mbar_wait(bar(B_ODONE + x), done[x] & 1u, abort_flag, p.status);
+        if (row == 0) TR(3, item_n, 3 + 5 * x);
         ++done[x];
         tc_fence_after();
         const float inv = inv_l[x * 128 + row];
@@ -561,6 +578,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         // the next item's first P V overwrites O, its softmax overwrites 1 / l: both wait for this
         tc_fence_before();
         mbar_arrive(bar(B_ODRAIN + x));
+        if (row == 0) TR(3, item_n, 4 + 5 * x);
       }
       it = nx;
     }
@@ -602,7 +620,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         fetch_item(item_n, it, true);
         if (it.n_tiles < 0) break;
         // Q tiles: free once the previous item's last S = Q K^T has completed
+        TR(4, item_n, 0);
         mbar_wait(bar(B_QEMPTY), (item_n & 1u) ^ 1u, abort_flag, p.status);
+        TR(4, item_n, 1);
         uint32_t rot_bytes = 0;
         const int pos_start = it.pos0 + it.tok0;
         if (ROT_SMEM) {
@@ -627,6 +647,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           // (gather mode: a route tile is filled by the epilogue warps; every stage barrier expects
           // their 128 arrivals plus one from here, whoever brings the data)
           mbar_wait(bar(B_KEMPTY + st), ph ^ 1u, abort_flag, p.status);
+          if (i == 0) TR(4, item_n, 2);
           if (GATHER && route) {
             mbar_arrive(bar(B_KFULL + st));
           } else {
@@ -642,6 +663,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             for (int kc = 0; kc < 2; ++kc)
               tma_load_2d(sm + SM_V + st * TILE_BYTES + kc * BOX_BYTES, route ? &tm_vr : &tm_vs, bar(B_VFULL + st), kc * 64, row);
           }
+          if (i == 0) TR(4, item_n, 3);
+          if (i == it.n_tiles - 1) TR(4, item_n, 4);
         }
       }
     }
@@ -687,16 +710,21 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       if (it.n_tiles < 0) break;
       const int n_tiles = it.n_tiles, nA = it.nA, lenA = it.lenA, L = it.H + it.L, kv_end = it.kv_end;
       const bool b_valid = it.b_valid != 0;
+      if (issuer) TR(2, item_n, 0);
       // each query tile starts as soon as its own half of Q has been rotated
       mbar_wait(bar(B_QREADY + 0), item_n & 1u, abort_flag, p.status);
+      if (issuer) TR(2, item_n, 1);
       mbar_wait(bar(B_KFULL + kv_n % NSTAGE), (kv_n / NSTAGE) & 1u, abort_flag, p.status);
+      if (issuer) TR(2, item_n, 2);
       if (GATHER) fence_async_smem();   // the tile may have been written by cp.async (generic proxy)
       tc_fence_after();
       const int st0 = kv_n % NSTAGE;
       if (issuer) { issue_qk(0, st0); tc_commit(bar(B_SFULL + 0)); }
       // (waited for even when the second tile is empty: its warps still rewrite that half of Q,
       // and the Q-empty commit below lets the next load overwrite it)
+      if (issuer) TR(2, item_n, 3);
       mbar_wait(bar(B_QREADY + 1), item_n & 1u, abort_flag, p.status);
+      if (issuer) TR(2, item_n, 4);
       tc_fence_after();
       if (issuer) {
         if (b_valid) { issue_qk(1, st0); tc_commit(bar(B_SFULL + 1)); }
@@ -712,6 +740,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const int vis_rows = i < nA ? seg_rows : kv_end - (i - nA) * TILE_N;
         const int ksteps = (min(vis_rows, TILE_N) + 15) >> 4;
         mbar_wait(bar(B_VFULL + st), ph, abort_flag, p.status);
+        if (issuer && i == 0) TR(2, item_n, 5);
         if (GATHER) fence_async_smem();
         if (seg_rows < ksteps * 16) {
           // rows past the segment hold whatever follows it in memory: zero them, 0 * NaN would poison O
@@ -729,7 +758,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const bool more = i + 1 < n_tiles;
         // P of keys 0..63 arrives first: half of P V runs while the softmax finishes the other half
         mbar_wait(bar(B_PHALF + 0), cnt[0] & 1u, abort_flag, p.status);
+        if (issuer && i == 0) TR(2, item_n, 6);
         if (i == 0 && items_x[0] > 0) mbar_wait(bar(B_ODRAIN + 0), (items_x[0] - 1u) & 1u, abort_flag, p.status);
+        if (issuer && i == 0) TR(2, item_n, 7);
         tc_fence_after();
         if (issuer) issue_pv(0, st, 0, min(ksteps, 4), i == 0);
         mbar_wait(bar(B_PREADY + 0), cnt[0]++ & 1u, abort_flag, p.status);
@@ -742,8 +773,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           if (issuer) { issue_qk(0, st1); tc_commit(bar(B_SFULL + 0)); }
         }
         if (b_valid) {
+          if (issuer && i == 0) TR(2, item_n, 8);
           mbar_wait(bar(B_PHALF + 1), cnt[1] & 1u, abort_flag, p.status);
+          if (issuer && i == 0) TR(2, item_n, 9);
           if (i == 0 && items_x[1] > 0) mbar_wait(bar(B_ODRAIN + 1), (items_x[1] - 1u) & 1u, abort_flag, p.status);
+          if (issuer && i == 0) TR(2, item_n, 10);
           tc_fence_after();
           if (issuer) issue_pv(1, st, 0, min(ksteps, 4), i == 0);
           mbar_wait(bar(B_PREADY + 1), cnt[1]++ & 1u, abort_flag, p.status);
@@ -759,7 +793,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           }
         }
         __syncwarp();
+        if (issuer && i == 0) TR(2, item_n, 11);
+        if (issuer && i == n_tiles - 2) TR(2, item_n, 12);
       }
+      if (issuer) { TR(2, item_n, 13); TRV(2, item_n, 15, n_tiles * 2 + (b_valid ? 1 : 0)); }
       kv_n += (uint32_t)n_tiles;
       ++items_x[0];
       if (b_valid) ++items_x[1];
@@ -782,7 +819,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     // time and goes through the token's s heads, so that cos / sin are read once per token, not
     // once per row; the 8 lanes of a token cover whole 128-byte rows of Q.
     auto rotate_q = [&](const Item& it, uint32_t n_item) {
+      if (row == 0) TR(x, n_item, 0);
       mbar_wait(bar(B_QFULL), n_item & 1u, abort_flag, p.status);
+      if (row == 0) TR(x, n_item, 1);
       uint8_t* qt = sm_gen + SM_Q + x * TILE_BYTES;
       for (int u = row; u < TQ * 8; u += 128) {
         const int tok = u >> 3, c = u & 7;
@@ -833,6 +872,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       }
       fence_async_smem();
       mbar_arrive(bar(B_QREADY + x));
+      if (row == 0) TR(x, n_item, 2);
     };
 
     Item it, nx;
@@ -848,6 +888,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       if (active) {
         for (int i = 0; i < n_tiles; ++i, ++cnt) {
           mbar_wait(bar(B_SFULL + x), cnt & 1u, abort_flag, p.status);
+          if (row == 0 && i == 0) TR(x, item_n, 3);
+          if (row == 0 && i == 1) TR(x, item_n, 5);
+          if (row == 0 && i == n_tiles - 1) TR(x, item_n, 6);
           tc_fence_after();
           if (releaser) {
             // S of tile i is complete: so is every earlier MMA, i.e. the last reader of K tile i
@@ -917,11 +960,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(bar(B_PREADY + x));
+          if (row == 0 && i == 0) TR(x, item_n, 4);
+          if (row == 0 && i == n_tiles - 1) TR(x, item_n, 7);
         }
       }
       // ---- hand the finished tile to the epilogue warps (they wait for its last P V themselves) ----
       if (active) {
         if (done_n > 0) mbar_wait(bar(B_ODRAIN + x), (done_n - 1u) & 1u, abort_flag, p.status);   // 1 / l of the item before was read
+        if (row == 0) TR(x, item_n, 8);
         reinterpret_cast<float*>(sm_gen + SM_INVL)[x * 128 + row] = 1.f / l_sum;
         mbar_arrive(bar(B_LREADY + x));
         ++done_n;
@@ -929,6 +975,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
       kv_n += (uint32_t)n_tiles;
       // ---- next item's Q (its load was issued a tile ago) ----
       fetch_item(item_n + 1, nx, true);
+      if (row == 0) { TR(x, item_n, 9); TRV(x, item_n, 15, n_tiles * 2 + it.b_valid); }
       if (nx.n_tiles > 0) rotate_q(nx, item_n + 1);
       it = nx; ++item_n;
     }
@@ -989,6 +1036,14 @@ bool map_q(CUtensorMap* m, const void* base, uint64_t tokens, int Hq, int s) {
 int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
 
 }  // namespace
+
+#ifdef RC_TRACE
+extern "C" __attribute__((visibility("default"))) int recache_debug_trace(long long* host, int n) {
+  const int m = TR_ROLES * TR_ITEMS * 16;
+  if (n < m) return -m;
+  return cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * m) == cudaSuccess ? m : -1;
+}
+#endif
 
 bool rc_tc_supported(const recache_ctx* ctx) {
   const int s = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;

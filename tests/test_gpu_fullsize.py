@@ -121,12 +121,13 @@ def test_bench_step_full_size():
         assert _close(f64(od[b, kg * s:(kg + 1) * s]), ref_o[0])
 
 
-def test_composition_reuse_full_size_layer():
-    """One layer of the composition-reuse workload at full size: a pool of 64
-    resources U[150,1200] encoded once, 16 requests of 4-12 pool resources in
-    random order with 256-1024 query tokens; sampled rows against the oracle and
-    exact compaction.  (The 36 layers differ only in their seeds and routes.)"""
-    layer = 7
+@pytest.mark.parametrize("layer", [0, 7, 35])
+def test_composition_reuse_full_size_layer(layer):
+    """Layers of the composition-reuse workload at full size (the first, one in
+    the middle, the last of the 36): a pool of 64 resources U[150,1200] encoded
+    once, 16 requests of 4-12 pool resources in random order with 256-1024 query
+    tokens; sampled rows against the oracle and exact compaction.  (The layers
+    differ in their inputs and routes.)"""
     pool = wl.config3_pool(layer=layer)
     sh = pool.shape
     req = wl.config3_requests(pool, layer=layer)
@@ -152,4 +153,34 @@ def test_composition_reuse_full_size_layer():
                             sh.rope_theta, prow, storage="bf16")
     pc = p.cpu()
     assert _close(np.stack([f64(pc[t, h]) for t, h in prow]), pref)
+    assert rc.poll_status() == 0
+
+
+def test_long_resource_bit_identical_across_work_list_orders():
+    """The encode launch orders its work two ways: the whole pool of 64 resources
+    makes thousands of work items and is walked sequence by sequence, a launch of
+    three resources is sorted heaviest-first.  A resource of more than 1000
+    tokens encoded in both gives the same output and cache rows, bit for bit."""
+    layer = 3
+    pool = wl.config3_pool(layer=layer)
+    sh = pool.shape
+    long_ids = [int(i) for i in np.argsort(-pool.lens)[:2]]
+    assert pool.lens[long_ids[1]] >= 1000
+    tpi = 2 * 128 // sh.group_size                      # tokens per work item
+    assert sum((int(n) + tpi - 1) // tpi for n in pool.lens) * sh.n_kv_heads > 1024      # sequence-major order
+    rc = make_ctx(sh, max_pos=16384)
+    o_all, kc, vc = gpu_encode(rc, pool, out_dtype=torch.bfloat16)
+    sub = [long_ids[0], int(np.argmin(pool.lens)), long_ids[1]]
+    assert sum((int(pool.lens[r]) + tpi - 1) // tpi for r in sub) * sh.n_kv_heads <= 1024  # sorted order
+    masks = [pool.keep[pool.dst_slot[r]:pool.dst_slot[r] + pool.lens[r]] for r in sub]
+    pool_b = wl.pack_resources(sh, wl.SEED0 + 3, pool.lens[sub], masks, res_ids=sub, layer=layer, slot_gap=11)
+    o_b, kc_b, vc_b = gpu_encode(rc, pool_b, out_dtype=torch.bfloat16)
+    for n, r in enumerate(sub):
+        a, e = pool.cu_seqlens[r], pool.cu_seqlens[r + 1]
+        a2, e2 = pool_b.cu_seqlens[n], pool_b.cu_seqlens[n + 1]
+        assert torch.equal(pool.q[a:e], pool_b.q[a2:e2])
+        assert torch.equal(o_all[a:e].view(torch.int16), o_b[a2:e2].view(torch.int16))
+        s1, s2, ln = pool.dst_slot[r], pool_b.dst_slot[n], pool.lens[r]
+        assert torch.equal(kc[:, s1:s1 + ln].view(torch.int16), kc_b[:, s2:s2 + ln].view(torch.int16))
+        assert torch.equal(vc[:, s1:s1 + ln].view(torch.int16), vc_b[:, s2:s2 + ln].view(torch.int16))
     assert rc.poll_status() == 0
