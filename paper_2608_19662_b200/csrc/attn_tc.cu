@@ -92,11 +92,22 @@ struct TcParams {
 #ifdef RC_TRACE
 constexpr int TR_ITEMS = 192, TR_ROLES = 5;   // roles: softmax A, softmax B, MMA, epilogue, producer
 __device__ long long g_trace[TR_ROLES * TR_ITEMS * 16];
-#define TR(role, item, k) do { if (blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = clock64(); } while (0)
-#define TRV(role, item, k, v) do { if (blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = (v); } while (0)
+#ifndef RC_TRACE_ROLES
+#define RC_TRACE_ROLES 31   // bit per role: stamping the 32-register roles disturbs them most
+#endif
+#define TR(role, item, k) do { if (((RC_TRACE_ROLES >> (role)) & 1) && blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = clock64(); } while (0)
+#define TRV(role, item, k, v) do { if (((RC_TRACE_ROLES >> (role)) & 1) && blockIdx.x == 0 && (item) < (uint32_t)TR_ITEMS) g_trace[((role) * TR_ITEMS + (item)) * 16 + (k)] = (v); } while (0)
 #else
 #define TR(role, item, k) do {} while (0)
 #define TRV(role, item, k, v) do {} while (0)
+#endif
+// A second, non-intrusive form (-DRC_OBSERVE): the otherwise idle warp 11 of CTA 0 polls the CTA's
+// barriers with test_wait and logs (clock, barrier) whenever one completes a phase, so the timeline
+// of the hand-overs is seen without a single extra instruction in the working roles.
+#ifdef RC_OBSERVE
+constexpr int OBS_PER = 2048;                 // events per barrier
+__device__ long long g_observe[32 * OBS_PER];   // row 31, entry 0: start time
+__device__ int g_observe_n[32];
 #endif
 
 // ------------------------------------------------------------------ PTX --
@@ -584,6 +595,32 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
   } else if (warp >= 8) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_AUX));
+#ifdef RC_OBSERVE
+  if (warp == 11 && blockIdx.x == 0) {
+    // lane b watches barrier b (lanes past the last barrier watch barrier 0 and log nothing)
+    const bool logs = lane < B_COUNT;
+    const uint32_t my = bar(logs ? lane : 0);
+    uint32_t par = 0;
+    int n = 0;
+    const long long start = clock64();
+    if (lane == 0) g_observe[OBS_PER * 31] = start;
+    uint32_t last = (uint32_t)start;
+    for (uint32_t iter = 0;; ++iter) {
+      uint32_t ok, now;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%2], %3;\n\tselp.u32 %0, 1, 0, p;\n\tmov.u32 %1, %%clock;\n\t}"
+                   : "=r"(ok), "=r"(now) : "r"(my), "r"(par) : "memory");
+      if (ok) {
+        par ^= 1u; last = now;
+        if (logs && n < OBS_PER) g_observe[lane * OBS_PER + n++] = start + (long long)(uint32_t)(now - (uint32_t)start);
+      }
+      if ((iter & 63u) == 63u) {
+        const uint32_t newest = __reduce_max_sync(0xffffffffu, last - (uint32_t)start);
+        if ((now - (uint32_t)start) - newest > 60000u) break;
+      }
+    }
+    if (logs) g_observe_n[lane] = n;
+  }
+#endif
   if (warp == 10) {
     // ===================== scheduler =====================
     if (lane == 0) {
@@ -1037,6 +1074,12 @@ int64_t align256(int64_t x) { return (x + 255) & ~(int64_t)255; }
 
 }  // namespace
 
+#ifdef RC_OBSERVE
+extern "C" __attribute__((visibility("default"))) int recache_debug_observe(long long* host, int* counts) {
+  if (cudaMemcpyFromSymbol(counts, g_observe_n, sizeof(int) * 32) != cudaSuccess) return -1;
+  return cudaMemcpyFromSymbol(host, g_observe, sizeof(long long) * 32 * OBS_PER) == cudaSuccess ? 32 * OBS_PER : -1;
+}
+#endif
 #ifdef RC_TRACE
 extern "C" __attribute__((visibility("default"))) int recache_debug_trace(long long* host, int n) {
   const int m = TR_ROLES * TR_ITEMS * 16;
