@@ -303,11 +303,13 @@ __device__ __forceinline__ bool load_item(const TcParams& p, int w, Item& it) {
 }
 
 // ------------------------------------------------------------- work list --
-// Items = (sequence, tile-pair index): sequence by sequence, and inside a
-// sequence the last (heaviest) tile pair first.  With the KV group as the
+// Items = (sequence, tile-pair index): sequence by sequence, the longest sequences
+// first, and inside a sequence the last (heaviest) tile pair first, so that the
+// launch ends on the light items of short sequences.  With the KV group as the
 // fastest index of the flattened work list, the CTAs that run at the same time
 // share one sequence's K/V, which then stays in L2 instead of being streamed
-// from HBM once per tile pair.  One CTA; level_off[b] = first item of sequence b.
+// from HBM once per tile pair.  One CTA.  (Sequences of equal length land in an
+// order that may differ between launches; no result depends on it.)
 __global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int tok_per_cta, int n_levels,
                                                          int2* __restrict__ items, int32_t* __restrict__ level_off,
                                                          int32_t* __restrict__ order, int max_items) {
@@ -348,12 +350,39 @@ __global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int t
       p.header[1] = 0;         // dynamic work counter of the attention kernel
     }
   }
+  // counting sort of the sequences by their number of tile pairs, longest first: hist[bin] = items of
+  // that bin, then (scanned from the top bin down) the first item index of the bin
+  for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
   __syncthreads();
-  int k = warp_sum[warp] + incl - sum;
   for (int b = b0; b < b1; ++b) {
     const int len = cu[b + 1] - cu[b];
     int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
     if (nt > n_levels) nt = n_levels;
+    if (nt > 0) atomicAdd(&hist[min(nt, 1024)], nt);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int c0 = 1024; c0 >= 0; c0 -= 32) {      // lane 0 takes the highest bin of the chunk
+      const int bin_i = c0 - lane;
+      const int v = bin_i >= 0 ? hist[bin_i] : 0;
+      int vi = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, vi, off);
+        if (lane >= off) vi += u;
+      }
+      if (bin_i >= 0) hist[bin_i] = carry + vi - v;
+      carry += __shfl_sync(0xffffffffu, vi, 31);
+    }
+  }
+  __syncthreads();
+  for (int b = b0; b < b1; ++b) {
+    const int len = cu[b + 1] - cu[b];
+    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+    if (nt > n_levels) nt = n_levels;
+    if (nt == 0) continue;
+    int k = atomicAdd(&hist[min(nt, 1024)], nt);
     level_off[b] = k;
     for (int l = nt - 1; l >= 0; --l, ++k)
       if (k < max_items) items[k] = make_int2(b, l);
