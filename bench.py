@@ -42,10 +42,10 @@ sys.path.insert(0, ROOT)
 from paper_2608_19662_b200 import workloads as wl  # noqa: E402
 
 # DRAM traffic of the encode attention launch from an ncu capture of the medium case
-# (dram__bytes_read.sum + dram__bytes_write.sum = 413.3 MB for 21,626 resource tokens).  The full
+# (dram__bytes_read.sum + dram__bytes_write.sum = 414.5 MB for 21,626 resource tokens).  The full
 # workload is too large for a multi-pass capture; traffic grows in proportion to the tokens (Q read,
 # O written, K/V read once from HBM and re-read from L2), so it is scaled per token.
-NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 413.339e6 / 21626
+NCU_ENCODE_DRAM_BYTES_PER_TOKEN = 414.519e6 / 21626
 
 # Used only when the box's measured peaks are missing (an earlier measurement on the same kind of GPU).
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
