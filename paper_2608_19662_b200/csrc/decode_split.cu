@@ -411,14 +411,18 @@ __global__ void __launch_bounds__(GATHER ? NTHREADS_GATHER : NTHREADS, 1) decode
   if (*abort_flag) rc_timeout_drain();   // a wait ran out: let the loads in flight land before the CTA ends
 }
 
-// Combines the splits of every (sequence, head): grid = batch * Hq, 32 threads x 4 dims.
+// Combines the splits of every (sequence, head): one warp per output row (32 lanes x 4 dims), eight
+// rows per CTA.
+constexpr int MERGE_ROWS = 8;
 template <typename TO>
-__global__ void __launch_bounds__(32) decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                          TO* __restrict__ out, int n_splits, int G, int Hq, int s) {
-  const int row = blockIdx.x;                 // b * Hq + head
+__global__ void __launch_bounds__(32 * MERGE_ROWS) decode_merge_kernel(const float* __restrict__ part_o,
+                                                                       const float* __restrict__ part_ml,
+                                                                       TO* __restrict__ out, int n_rows, int n_splits, int G, int Hq, int s) {
+  const int row = blockIdx.x * MERGE_ROWS + (threadIdx.x >> 5);   // b * Hq + head
+  if (row >= n_rows) return;
   const int b = row / Hq, head = row % Hq, g = head / s, h = head % s;
   const int it = b * G + g;
-  const int t = threadIdx.x;
+  const int t = threadIdx.x & 31;
   float M = -INFINITY;
   for (int sp = 0; sp < n_splits; ++sp) M = fmaxf(M, part_ml[((int64_t)(it * n_splits + sp) * s + h) * 2]);
   float L = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -538,8 +542,9 @@ cudaError_t rc_launch_decode_split(const recache_ctx* ctx, const DecodeArgs& a, 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || ns == 1) return e;
   RcLaunchScope scope(ctx, RC_K_DECODE_MERGE, st);
-  if (f32) decode_merge_kernel<float><<<a.batch * Hq, 32, 0, st>>>(p.part_o, p.part_ml, (float*)a.o, ns, G, Hq, s);
-  else decode_merge_kernel<__nv_bfloat16><<<a.batch * Hq, 32, 0, st>>>(p.part_o, p.part_ml, (__nv_bfloat16*)a.o, ns, G, Hq, s);
+  const int n_rows = a.batch * Hq, blocks = (n_rows + MERGE_ROWS - 1) / MERGE_ROWS;
+  if (f32) decode_merge_kernel<float><<<blocks, 32 * MERGE_ROWS, 0, st>>>(p.part_o, p.part_ml, (float*)a.o, n_rows, ns, G, Hq, s);
+  else decode_merge_kernel<__nv_bfloat16><<<blocks, 32 * MERGE_ROWS, 0, st>>>(p.part_o, p.part_ml, (__nv_bfloat16*)a.o, n_rows, ns, G, Hq, s);
   return cudaGetLastError();
 }
 
