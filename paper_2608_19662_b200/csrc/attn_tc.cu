@@ -350,50 +350,64 @@ __global__ void __launch_bounds__(1024) tile_plan_kernel(const TcParams p, int t
       p.header[1] = 0;         // dynamic work counter of the attention kernel
     }
   }
-  // counting sort of the sequences by their number of tile pairs, longest first: hist[bin] = items of
-  // that bin, then (scanned from the top bin down) the first item index of the bin
-  for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
   __syncthreads();
-  for (int b = b0; b < b1; ++b) {
-    const int len = cu[b + 1] - cu[b];
-    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
-    if (nt > n_levels) nt = n_levels;
-    if (nt > 0) atomicAdd(&hist[min(nt, 1024)], nt);
-  }
-  __syncthreads();
-  if (warp == 0) {
-    int carry = 0;
-    for (int c0 = 1024; c0 >= 0; c0 -= 32) {      // lane 0 takes the highest bin of the chunk
-      const int bin_i = c0 - lane;
-      const int v = bin_i >= 0 ? hist[bin_i] : 0;
-      int vi = v;
-#pragma unroll
-      for (int off = 1; off < 32; off <<= 1) {
-        const int u = __shfl_up_sync(0xffffffffu, vi, off);
-        if (lane >= off) vi += u;
-      }
-      if (bin_i >= 0) hist[bin_i] = carry + vi - v;
-      carry += __shfl_sync(0xffffffffu, vi, 31);
+  // (an encode launch shares K/V between the items of a sequence only: beyond a thousand items the
+  // sequence-major order, which keeps a sequence's K/V in L2, is worth more than the balance)
+  const int n_work = p.header[0] * p.G;
+  const bool sorted = n_work <= (p.route_cu ? SORT_MAX : SORT_MAX / 4);
+  if (sorted) {
+    // few work items: they are sorted one by one below, so the sequences keep their order here
+    int k = warp_sum[warp] + incl - sum;
+    for (int b = b0; b < b1; ++b) {
+      const int len = cu[b + 1] - cu[b];
+      int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+      if (nt > n_levels) nt = n_levels;
+      level_off[b] = k;
+      for (int l = nt - 1; l >= 0; --l, ++k)
+        if (k < max_items) items[k] = make_int2(b, l);
     }
-  }
-  __syncthreads();
-  for (int b = b0; b < b1; ++b) {
-    const int len = cu[b + 1] - cu[b];
-    int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
-    if (nt > n_levels) nt = n_levels;
-    if (nt == 0) continue;
-    int k = atomicAdd(&hist[min(nt, 1024)], nt);
-    level_off[b] = k;
-    for (int l = nt - 1; l >= 0; --l, ++k)
-      if (k < max_items) items[k] = make_int2(b, l);
+  } else {
+    // counting sort of the sequences by their number of tile pairs, longest first: hist[bin] = items of
+    // that bin, then (scanned from the top bin down) the first item index of the bin
+    for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (int b = b0; b < b1; ++b) {
+      const int len = cu[b + 1] - cu[b];
+      int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+      if (nt > n_levels) nt = n_levels;
+      if (nt > 0) atomicAdd(&hist[min(nt, 1024)], nt);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      int carry = 0;
+      for (int c0 = 1024; c0 >= 0; c0 -= 32) {      // lane 0 takes the highest bin of the chunk
+        const int bin_i = c0 - lane;
+        const int v = bin_i >= 0 ? hist[bin_i] : 0;
+        int vi = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, vi, off);
+          if (lane >= off) vi += u;
+        }
+        if (bin_i >= 0) hist[bin_i] = carry + vi - v;
+        carry += __shfl_sync(0xffffffffu, vi, 31);
+      }
+    }
+    __syncthreads();
+    for (int b = b0; b < b1; ++b) {
+      const int len = cu[b + 1] - cu[b];
+      int nt = len > 0 ? (len + tok_per_cta - 1) / tok_per_cta : 0;
+      if (nt > n_levels) nt = n_levels;
+      if (nt == 0) continue;
+      int k = atomicAdd(&hist[min(nt, 1024)], nt);
+      level_off[b] = k;
+      for (int l = nt - 1; l >= 0; --l, ++k)
+        if (k < max_items) items[k] = make_int2(b, l);
+    }
   }
   // Few work items (a prefill of a handful of requests): one CTA gets one or two of them, so their
   // order decides the tail.  Sort them by weight (K/V tiles), heaviest first, with a counting sort.
   __syncthreads();
-  const int n_work = p.header[0] * p.G;
-  // (an encode launch shares K/V between the items of a sequence only: beyond a thousand items the
-  // sequence-major order, which keeps a sequence's K/V in L2, is worth more than the balance)
-  const bool sorted = n_work <= (p.route_cu ? SORT_MAX : SORT_MAX / 4);
   if (threadIdx.x == 0) p.header[2] = sorted ? 1 : 0;
   if (!sorted) return;
   for (int i = threadIdx.x; i < 1025; i += blockDim.x) hist[i] = 0;
