@@ -184,3 +184,46 @@ def test_long_resource_bit_identical_across_work_list_orders():
         assert torch.equal(kc[:, s1:s1 + ln].view(torch.int16), kc_b[:, s2:s2 + ln].view(torch.int16))
         assert torch.equal(vc[:, s1:s1 + ln].view(torch.int16), vc_b[:, s2:s2 + ln].view(torch.int16))
     assert rc.poll_status() == 0
+
+
+def test_dense_comparison_full_size_sampled_rows():
+    """The comparison point of the long-tool-set workload at full size: every
+    route sees every token of all 64 resources (keep-all masks), 2048 query
+    tokens over ~95k rows per group.  Exact compaction (identity ranges) and
+    sampled prefill rows against the oracle."""
+    pool, req = wl.config5()
+    pool, req = wl.keep_all(pool), wl.all_visible(req)
+    sh = pool.shape
+    g, d = sh.n_kv_heads, sh.head_dim
+    rc = make_ctx(sh, max_pos=int(req.q_pos0.max() + req.max_q) + 1)
+    kc = wl.seeded_normal(91, (g, pool.pool_tokens, d), sh.torch_dtype, device="cuda")    # stand-in for an earlier encode
+    vc = wl.seeded_normal(92, (g, pool.pool_tokens, d), sh.torch_dtype, device="cuda")
+    out = gpu_compact(rc, pool, req, kc, vc)
+    cu = out["route_cu"].cpu().numpy()
+    n = pool.total_tokens
+    assert np.array_equal(cu, np.arange(g + 1) * n)                       # every group holds every token
+    want = np.concatenate([np.arange(s0, s0 + ln) for s0, ln in zip(req.res_slot, req.res_len)])
+    idx = out["route_idx"].cpu().numpy()
+    for kg in range(g):
+        assert np.array_equal(idx[kg * n:(kg + 1) * n], want)
+    p, _, _ = gpu_prefill(rc, req, out["k_out"], out["v_out"], out["route_cu"], out_dtype=torch.bfloat16)
+    rng = np.random.default_rng(55)
+    prow = sample_rows(rng, req.cu_q, sh.n_q_heads, 48, extra_tokens=[31, 32, 63, 64, 1023, 1024])
+    rows = [[want.astype(np.int32) for _ in range(g)]]
+    f32 = lambda t: t.float().numpy()
+    kc_h, vc_h = kc.cpu().float().numpy(), vc.cpu().float().numpy()        # bf16 values are exact in fp32
+    pref = orc.prefill_rows(f32(req.q), f32(req.k_conv), f32(req.v_conv), req.cu_q, req.q_pos0, rows, kc_h, vc_h,
+                            sh.rope_theta, prow, storage="bf16")
+    pc = p.cpu()
+    assert _close(np.stack([f64(pc[t, h]) for t, h in prow]), pref)
+    assert rc.poll_status() == 0
+
+
+def test_bench_composition_reuse_stack_runs():
+    """The benchmark's 36-layer composition-reuse stack, cut to two layers: runs through the public calls with
+    a clean status word and reports plausible work and rates."""
+    import bench
+    peaks, _ = bench.load_peaks()
+    r = bench.other_workload_config3_stack(0, peaks, n_layers=2, reps=1)
+    assert r["useful_tflop_per_stack"] > 0.5 and r["ms_per_stack"] > 0
+    assert 50 < r["encode_attn"]["tflops"] < 2300 and 50 < r["prefill_attn"]["tflops"] < 2300
